@@ -1,0 +1,106 @@
+"""The five benchmark/parity workloads as data, plus the tensors of one layer.
+
+Shapes are the linear layers of Gemma2-2B and Llama3.1-8B (the models of the
+paper's Section 4.2 tables) under the 8/4/4 scheme: int8 per-channel for the
+attention projections, int4 for the feed-forward layers and the LM head; the
+int4 weights use group size 32 along K.  All tensors are synthetic (see
+generators.py); there is no arithmetic of the linear layer in this module.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+from . import generators as gen
+
+BASE_SEED = 2505002320  # config c (1-based) uses BASE_SEED + c
+
+
+@dataclass(frozen=True)
+class LayerSpec:
+    name: str
+    N: int          # output channels (rows of W)
+    K: int          # input channels (columns of W)
+    bits: int       # 4 or 8
+    group: int      # 0 = one scale per output channel, else group size along K
+    lo: int         # integer range, closed
+    hi: int
+
+    @property
+    def n_groups(self) -> int:
+        return 1 if self.group == 0 else self.K // self.group
+
+    @property
+    def weight_bytes(self) -> int:
+        """Algorithmic bytes streamed per forward call: packed integers + fp16 scales."""
+        return self.N * self.K * self.bits // 8 + 2 * self.N * self.n_groups
+
+    def flops(self, M: int) -> int:
+        return 2 * M * self.N * self.K
+
+
+def _i8(name, N, K, lo=-128, hi=127):
+    return LayerSpec(name, N, K, 8, 0, lo, hi)
+
+
+def _i4(name, N, K):
+    return LayerSpec(name, N, K, 4, 32, -8, 7)
+
+
+GEMMA2_2B = (
+    _i8("q", 2048, 2304), _i8("k", 1024, 2304), _i8("v", 1024, 2304), _i8("o", 2304, 2048),
+    _i4("gate", 9216, 2304), _i4("up", 9216, 2304), _i4("down", 2304, 9216),
+)
+LLAMA31_8B = (
+    _i8("q", 4096, 4096), _i8("k", 1024, 4096), _i8("v", 1024, 4096), _i8("o", 4096, 4096),
+    _i4("gate", 14336, 4096), _i4("up", 14336, 4096), _i4("down", 4096, 14336),
+)
+LLAMA31_8B_HEAD = _i4("lm_head", 128256, 4096)
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    index: int               # 1-based config number
+    layers: tuple
+    Ms: tuple                # token counts the config is run at
+    stage: str               # "decode" or "prefill"
+
+    @property
+    def seed(self) -> int:
+        return BASE_SEED + self.index
+
+
+CONFIGS = (
+    Workload("int8_gemv_2304", 1, (_i8("fc", 2304, 2304, -127, 127),), (1,), "decode"),
+    Workload("gemma2_2b_decode", 2, GEMMA2_2B, (1,), "decode"),
+    Workload("llama31_8b_decode", 3, LLAMA31_8B, (1, 4), "decode"),
+    Workload("gemma2_2b_prefill", 4, tuple(l for l in GEMMA2_2B if l.bits == 4), (1024,), "prefill"),
+    Workload("llama31_8b_prefill", 5, LLAMA31_8B, (2048,), "prefill"),
+)
+CONFIG_5B = Workload("llama31_8b_lm_head", 5, (LLAMA31_8B_HEAD,), (1,), "decode")
+
+
+def by_name(name: str) -> Workload:
+    for w in CONFIGS + (CONFIG_5B,):
+        if w.name == name:
+            return w
+    raise KeyError(name)
+
+
+def tensor_id(copy: int, layer_index: int, kind: str) -> int:
+    """Stream id of one tensor: (weight copy, layer within the workload, 'q' | 's' | 'x')."""
+    return (copy * 64 + layer_index) * 4 + {"q": 0, "s": 1, "x": 2}[kind]
+
+
+def layer_weights(seed: int, layer: LayerSpec, layer_index: int = 0, copy: int = 0):
+    """(q, s): q int8 [N, K] one integer per byte; s fp16 [N, n_groups]."""
+    q = gen.uniform_ints(seed, tensor_id(copy, layer_index, "q"), (layer.N, layer.K), layer.lo, layer.hi)
+    s = gen.uniform_scales_fp16(seed, tensor_id(copy, layer_index, "s"), (layer.N, layer.n_groups))
+    return q, s
+
+
+def layer_activations(seed: int, layer: LayerSpec, M: int, layer_index: int = 0) -> np.ndarray:
+    """x fp16 [M, K] ~ N(0, 1)."""
+    return gen.normal_fp16(seed, tensor_id(0, layer_index, "x"), (M, layer.K))
