@@ -1,0 +1,119 @@
+/*
+ * qlinear -- weight-only quantised linear layer for NVIDIA B200 (sm_100a).
+ *
+ *     y[m,n] = fp16( sum_k x[m,k] * s[n, k/G] * q[n,k] )        fp32 accumulation
+ *
+ * W = s*q is N x K (output channels x input channels: the O x I weight
+ * orientation of the paper's Section 3.1), q are int8 or int4 integers, s are
+ * fp16 scales (one per output channel, or one per group of G consecutive k),
+ * x is M x K fp16 row-major, y is M x N fp16 row-major.
+ *
+ * The calls follow the life cycle the paper describes for operators with
+ * external weights: the weights are converted once, at initialisation, into the
+ * memory layout the kernels read (Section 3.4, "weights conversion"; Section
+ * 3.1, weight layouts); every forward call then picks the kernel for its stage
+ * from the shape of the input (Section 3.7: a memory-bound fully-connected
+ * kernel for decode, a compute-bound matrix-multiply kernel for prefill), both
+ * reading the same resident weights.  Quantisation schemes: Section 4.2 (q8 =
+ * int8 per channel; 8/4/4 = int8 attention, int4 feed-forward/embedding).
+ *
+ * All functions are thread-safe; a handle is immutable after creation.  No
+ * function falls back to the CPU: without an sm_100 device qlinear_create
+ * fails with QL_ERR_ARCH.
+ */
+#ifndef QLINEAR_H
+#define QLINEAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qlinear_s* qlinear_t;
+
+typedef enum {
+    QL_OK = 0,
+    QL_ERR_INVALID_ARG = 1,     /* null pointer, misaligned pointer, bad size, value out of range   */
+    QL_ERR_UNSUPPORTED = 2,     /* shape / bits / group combination the library does not implement   */
+    QL_ERR_ALLOC = 3,           /* host allocation failed                                            */
+    QL_ERR_CUDA = 4,            /* a CUDA runtime / driver call failed (launch errors included)      */
+    QL_ERR_DEVICE_TIMEOUT = 5,  /* a bounded wait inside a kernel expired; the output is invalid     */
+    QL_ERR_ARCH = 6             /* the device is not compute capability 10.x                         */
+} ql_status;
+
+/* Shape and quantisation scheme of one layer (Section 4.2).
+ *   N, K   output / input channels.  K must be a multiple of 32, N a multiple of 8.
+ *   bits   8 or 4.
+ *   group  0 = one scale per output channel; for bits == 4 also 32, 64 or 128 = scales per group of
+ *          that many consecutive k (must divide K).  bits == 8 supports group == 0 only. */
+typedef struct {
+    int32_t N, K, bits, group;
+} qlinear_desc;
+
+/* Which kernel a forward call with M tokens runs (Section 3.7, stage-aware selection). */
+typedef enum { QL_PATH_GEMV = 1, QL_PATH_GEMM = 2 } ql_path;
+
+/* Bytes of the packed blob for this layer; 0 if the descriptor is invalid or unsupported. */
+size_t qlinear_packed_size(const qlinear_desc* desc);
+
+/* Weights conversion (Section 3.4; layouts: Section 3.1).  HOST function, pure, calls no CUDA.
+ *   q        host, N*K int8, row-major, one integer per byte: [-128,127] for bits 8, [-8,7] for bits 4.
+ *   s_fp16   host, fp16 bit patterns, row-major [N] (group 0) or [N, K/group].
+ *   packed   host, out, packed_bytes >= qlinear_packed_size(desc).  Opaque, position-independent,
+ *            starts with a versioned header; the caller copies it to device memory unchanged.
+ * Errors: QL_ERR_INVALID_ARG (null, short buffer, integer outside the range of `bits`),
+ *         QL_ERR_UNSUPPORTED (descriptor). Nothing is written on error. */
+ql_status qlinear_pack(const qlinear_desc* desc, const int8_t* q, const uint16_t* s_fp16,
+                       void* packed, size_t packed_bytes);
+
+/* Host inverse of qlinear_pack (for tests and for re-exporting weights): fills q_out [N*K] and
+ * s_out [N] or [N, K/group].  Checks the header against desc (QL_ERR_INVALID_ARG on mismatch). */
+ql_status qlinear_unpack(const qlinear_desc* desc, const void* packed, int8_t* q_out, uint16_t* s_out);
+
+/* Binds a packed blob that already lives in DEVICE memory to a handle (Section 3.4: the converted
+ * weights stay resident in GPU memory and serve both stages, Section 3.7).
+ *   packed_dev  device pointer, 256-byte aligned, qlinear_packed_size(desc) bytes, owned by the caller,
+ *               must stay alive and unchanged until qlinear_destroy.
+ *   device      CUDA device ordinal that owns packed_dev.
+ * The handle owns host memory only.  Errors: QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ARCH
+ * (device is not sm_100), QL_ERR_CUDA, QL_ERR_ALLOC. */
+ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int device, qlinear_t* out);
+
+/* y = x . W^T for M >= 1 tokens, enqueued on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ *   x_dev  device, fp16 [M, K] row-major contiguous, 16-byte aligned, read-only during the call.
+ *   y_dev  device, fp16 [M, N] row-major contiguous, 16-byte aligned, must not overlap x_dev.
+ * Asynchronous: returns after the launch; allocates nothing; never synchronises.  M <= 8 runs the
+ * decode kernel, larger M the prefill kernel (Section 3.7); see qlinear_path_for.
+ * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, M < 1, M*K or M*N beyond 2^31-1 elements),
+ * QL_ERR_CUDA (launch failure, reported synchronously), QL_ERR_DEVICE_TIMEOUT (a previous call on this
+ * handle hit a bounded wait; see qlinear_device_status). */
+ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
+
+/* The kernel qlinear_forward uses for M tokens on this handle (0 if h is NULL or M < 1). */
+int32_t qlinear_path_for(qlinear_t h, int32_t M);
+
+/* Runs, on the device, the same unpack routine the forward kernels use and writes the integers
+ * q_dev_out [N*K] int8 row-major (device memory, caller-owned).  Used to prove that the device sees
+ * exactly the integers that were packed.  Asynchronous on `cuda_stream`. */
+ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_dev_out, void* cuda_stream);
+
+/* Synchronises the handle's device and reports whether any kernel launched through it gave up a
+ * bounded wait (QL_ERR_DEVICE_TIMEOUT), else QL_OK.  `detail`, if not NULL, receives a code that
+ * identifies the wait.  Clears the condition. */
+ql_status qlinear_device_status(qlinear_t h, uint32_t* detail);
+
+/* Frees the handle's host memory.  Does not touch the packed blob.  NULL is allowed. */
+ql_status qlinear_destroy(qlinear_t h);
+
+/* Static, NUL-terminated description of a status code. */
+const char* qlinear_status_string(ql_status s);
+
+/* Library ABI version (major << 16 | minor). */
+uint32_t qlinear_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QLINEAR_H */

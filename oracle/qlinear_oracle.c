@@ -24,6 +24,7 @@
  */
 #include <stdint.h>
 #include <string.h>
+#include <stdlib.h>
 #include <math.h>
 #ifdef _OPENMP
 #include <omp.h>
@@ -90,6 +91,9 @@ void oracle_dequantize(const int8_t* q, const uint16_t* s, int32_t N, int32_t K,
 void oracle_linear(const uint16_t* x, const double* w, int32_t M, int32_t N, int32_t K,
                    double* y64, double* A, uint16_t* y16)
 {
+    double* xd = (double*)malloc(sizeof(double) * (size_t)M * (size_t)K);   /* fp16 -> fp64, exact */
+    if (!xd) return;
+    for (int64_t i = 0; i < (int64_t)M * K; ++i) xd[i] = oracle_fp16_to_double(x[i]);
 #ifdef _OPENMP
 #pragma omp parallel for schedule(static)
 #endif
@@ -97,7 +101,7 @@ void oracle_linear(const uint16_t* x, const double* w, int32_t M, int32_t N, int
         for (int32_t m = 0; m < M; ++m) {
             double acc = 0.0, abs_acc = 0.0;
             for (int32_t k = 0; k < K; ++k) {
-                double p = oracle_fp16_to_double(x[(int64_t)m * K + k]) * w[(int64_t)n * K + k];
+                double p = xd[(int64_t)m * K + k] * w[(int64_t)n * K + k];
                 acc += p;
                 abs_acc += fabs(p);
             }
@@ -107,6 +111,7 @@ void oracle_linear(const uint16_t* x, const double* w, int32_t M, int32_t N, int
             if (y16) y16[o] = oracle_double_to_fp16(acc);
         }
     }
+    free(xd);
 }
 
 /* Threads oracle_linear uses (1 when built without OpenMP). */

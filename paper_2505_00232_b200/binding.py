@@ -1,0 +1,205 @@
+"""Thin ctypes binding over libqlinear.so (see include/qlinear.h): argument marshalling only.
+
+Every arithmetic step runs inside the library's CUDA kernels (or, for pack/unpack, its host
+packer).  torch is used for device memory and streams.  There is no CPU fallback: if the shared
+library has not been built, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqlinear.so")
+
+QL_OK = 0
+QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ALLOC, QL_ERR_CUDA, QL_ERR_DEVICE_TIMEOUT, QL_ERR_ARCH = 1, 2, 3, 4, 5, 6
+QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
+
+EXPORTS = (
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward",
+    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_destroy",
+    "qlinear_status_string", "qlinear_version",
+)
+
+
+class QLinearError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (ql_status {status})")
+
+
+class qlinear_desc(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int32), ("K", ctypes.c_int32), ("bits", ctypes.c_int32), ("group", ctypes.c_int32)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2505_00232_b200.build` "
+            "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32 = ctypes.c_void_p, ctypes.c_int32
+    dp = ctypes.POINTER(qlinear_desc)
+    lib.qlinear_packed_size.argtypes = [dp]
+    lib.qlinear_packed_size.restype = ctypes.c_size_t
+    lib.qlinear_pack.argtypes = [dp, vp, vp, vp, ctypes.c_size_t]
+    lib.qlinear_pack.restype = ctypes.c_int
+    lib.qlinear_unpack.argtypes = [dp, vp, vp, vp]
+    lib.qlinear_unpack.restype = ctypes.c_int
+    lib.qlinear_create.argtypes = [dp, vp, ctypes.c_int, ctypes.POINTER(vp)]
+    lib.qlinear_create.restype = ctypes.c_int
+    lib.qlinear_forward.argtypes = [vp, vp, vp, i32, vp]
+    lib.qlinear_forward.restype = ctypes.c_int
+    lib.qlinear_path_for.argtypes = [vp, i32]
+    lib.qlinear_path_for.restype = i32
+    lib.qlinear_debug_unpack_device.argtypes = [vp, vp, vp]
+    lib.qlinear_debug_unpack_device.restype = ctypes.c_int
+    lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.qlinear_device_status.restype = ctypes.c_int
+    lib.qlinear_destroy.argtypes = [vp]
+    lib.qlinear_destroy.restype = ctypes.c_int
+    lib.qlinear_status_string.argtypes = [ctypes.c_int]
+    lib.qlinear_status_string.restype = ctypes.c_char_p
+    lib.qlinear_version.restype = ctypes.c_uint32
+    return lib
+
+
+lib = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.qlinear_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != QL_OK:
+        raise QLinearError(status, where)
+
+
+def _np_ptr(a: np.ndarray) -> ctypes.c_void_p:
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+@dataclass(frozen=True)
+class Desc:
+    N: int
+    K: int
+    bits: int
+    group: int = 0
+
+    def c(self) -> qlinear_desc:
+        return qlinear_desc(self.N, self.K, self.bits, self.group)
+
+    @property
+    def n_groups(self) -> int:
+        return 1 if self.group == 0 else self.K // self.group
+
+
+# ---------------------------------------------------------------------------- host calls
+def qlinear_packed_size(desc: Desc) -> int:
+    return int(lib.qlinear_packed_size(ctypes.byref(desc.c())))
+
+
+def qlinear_pack(desc: Desc, q: np.ndarray, s: np.ndarray) -> np.ndarray:
+    """q int8 [N, K] (one integer per byte), s fp16 [N] or [N, K/group] -> packed blob (uint8 array)."""
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    s = np.ascontiguousarray(s, dtype=np.float16)
+    size = qlinear_packed_size(desc)
+    if size == 0:
+        raise QLinearError(QL_ERR_UNSUPPORTED, "qlinear_packed_size")
+    if q.shape != (desc.N, desc.K) or s.size != desc.N * desc.n_groups:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_pack (shape)")
+    out = np.empty(size, dtype=np.uint8)
+    _check(lib.qlinear_pack(ctypes.byref(desc.c()), _np_ptr(q), _np_ptr(s), _np_ptr(out), size), "qlinear_pack")
+    return out
+
+
+def qlinear_unpack(desc: Desc, packed: np.ndarray):
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    if packed.size < qlinear_packed_size(desc) or qlinear_packed_size(desc) == 0:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_unpack (size)")
+    q = np.empty((desc.N, desc.K), dtype=np.int8)
+    s = np.empty((desc.N, desc.n_groups), dtype=np.float16)
+    _check(lib.qlinear_unpack(ctypes.byref(desc.c()), _np_ptr(packed), _np_ptr(q), _np_ptr(s)), "qlinear_unpack")
+    return q, s
+
+
+# ---------------------------------------------------------------------------- device calls
+def _stream_ptr(stream) -> ctypes.c_void_p:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class QLinear:
+    """One quantised linear layer resident on a GPU: owns the packed device tensor and the handle."""
+
+    def __init__(self, desc: Desc, packed, device=None):
+        import torch
+        self.desc = desc
+        if isinstance(packed, np.ndarray):
+            dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+            packed = torch.from_numpy(np.ascontiguousarray(packed, dtype=np.uint8)).to(dev)
+        if not packed.is_cuda or packed.dtype != torch.uint8 or not packed.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "QLinear (packed must be a contiguous uint8 CUDA tensor)")
+        if packed.numel() < qlinear_packed_size(desc):
+            raise QLinearError(QL_ERR_INVALID_ARG, "QLinear (packed blob too small)")
+        self.packed = packed                      # keeps the device memory alive
+        self.device = packed.device
+        h = ctypes.c_void_p()
+        _check(lib.qlinear_create(ctypes.byref(desc.c()), ctypes.c_void_p(packed.data_ptr()),
+                                  self.device.index or 0, ctypes.byref(h)), "qlinear_create")
+        self._h = h
+
+    @classmethod
+    def from_weights(cls, q: np.ndarray, s: np.ndarray, bits: int, group: int = 0, device=None) -> "QLinear":
+        desc = Desc(int(q.shape[0]), int(q.shape[1]), bits, group)
+        return cls(desc, qlinear_pack(desc, q, s), device)
+
+    def forward(self, x, out=None, stream=None):
+        """x: fp16 CUDA tensor [M, K] -> y fp16 [M, N] (qlinear_forward on the current stream)."""
+        import torch
+        if x.dim() != 2 or x.shape[1] != self.desc.K or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward (x must be contiguous fp16 CUDA [M, K])")
+        M = x.shape[0]
+        if out is None:
+            out = torch.empty((M, self.desc.N), dtype=torch.float16, device=x.device)
+        elif out.shape != (M, self.desc.N) or out.dtype != torch.float16 or not out.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward (bad out tensor)")
+        self.forward_raw(x.data_ptr(), out.data_ptr(), M, stream)
+        return out
+
+    def forward_raw(self, x_ptr: int, y_ptr: int, M: int, stream=None) -> None:
+        _check(lib.qlinear_forward(self._h, ctypes.c_void_p(x_ptr), ctypes.c_void_p(y_ptr), M, _stream_ptr(stream)),
+               "qlinear_forward")
+
+    def path_for(self, M: int) -> int:
+        return int(lib.qlinear_path_for(self._h, M))
+
+    def debug_unpack(self, stream=None):
+        import torch
+        q = torch.empty((self.desc.N, self.desc.K), dtype=torch.int8, device=self.device)
+        _check(lib.qlinear_debug_unpack_device(self._h, ctypes.c_void_p(q.data_ptr()), _stream_ptr(stream)),
+               "qlinear_debug_unpack_device")
+        return q
+
+    def device_status(self):
+        detail = ctypes.c_uint32(0)
+        st = lib.qlinear_device_status(self._h, ctypes.byref(detail))
+        return int(st), int(detail.value)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            lib.qlinear_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

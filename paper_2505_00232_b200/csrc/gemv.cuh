@@ -1,0 +1,227 @@
+// Decode kernel: y = x . W^T for M <= 8 tokens (paper Section 3.7: the memory-bound decode stage is
+// served by a fully-connected kernel; Section 4.2: decode speed follows the weight bytes streamed).
+//
+// Work decomposition: a warp owns one row-block (16 output channels) and one K slice.  Per chunk it
+// issues one 16-byte load per lane (512 contiguous bytes per warp), unpacks in registers and feeds
+// mma.m16n8k16 with the weights as the 16-row operand and the <= 8 tokens as the 8 columns, so the
+// fp32 accumulation and the cross-lane part of the K reduction happen inside the tensor core.  The
+// K slices of a row-block are reduced across the warps of a CTA through shared memory and, when the
+// split is wider than one CTA, across the CTAs of a thread-block cluster through distributed shared
+// memory, always in a fixed order (deterministic, no atomics, no global scratch).
+//
+// Weight loads do not depend on the previous kernel in the stream, so the first batch is issued
+// before griddepcontrol.wait; with programmatic dependent launch the load ramp of this kernel then
+// overlaps the tail of the previous one.
+#pragma once
+#include <cooperative_groups.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dequant.cuh"
+#include "layout.h"
+
+namespace ql {
+namespace cg = cooperative_groups;
+
+constexpr int kGemvWarps = 8;
+constexpr int kGemvThreads = kGemvWarps * 32;
+constexpr int kGemvUnroll = 4;           // chunks in flight per lane per batch
+
+struct GemvParams {
+    const uint8_t* body;                 // first block of the packed body
+    const __half* chan_scales;           // per-channel scales (nullptr when grouped)
+    const __half* x;                     // [M, K]
+    __half* y;                           // [M, N]
+    int32_t M, N, K;
+    int32_t n_rb;                        // row-blocks holding at least one real row
+    int32_t n_kc;                        // chunks along K
+    int32_t block_bytes;
+    int32_t ks_cta;                      // K slices handled inside one CTA: 1, 2, 4 or 8
+    int32_t cl;                          // CTAs per cluster along K (1 = no cluster)
+    int32_t cps;                         // chunks per slice
+    int32_t x_stride;                    // halves between tokens in the shared x slab
+};
+
+__device__ __forceinline__ uint4 ldg_stream_v4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ uint2 ldg_stream_v2(const void* p)
+{
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void mma_16816(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+template <bool GROUPED>
+struct GemvBatch {
+    uint4 w[kGemvUnroll];
+    uint2 s[GROUPED ? kGemvUnroll : 1];
+};
+
+template <int BITS, bool GROUPED>
+__global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const GemvParams p)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __half* xs = reinterpret_cast<__half*>(smem_raw);                   // [M][x_stride]
+    __shared__ float red[kGemvWarps][128];
+    __shared__ float part[128];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, c = lane & 3;
+    constexpr int CHUNK_K = BITS == 4 ? 64 : 32;
+
+    const int crank = p.cl > 1 ? (int)(blockIdx.x % p.cl) : 0;
+    const int rb_group = p.cl > 1 ? (int)(blockIdx.x / p.cl) : (int)blockIdx.x;
+    const int rb_per_cta = kGemvWarps / p.ks_cta;
+    const int ks_local = warp % p.ks_cta;
+    const int rb = rb_group * rb_per_cta + warp / p.ks_cta;
+    const bool rb_live = rb < p.n_rb;
+    const int ks = crank * p.ks_cta + ks_local;
+    const int kc0 = min(ks * p.cps, p.n_kc);
+    const int kc1 = rb_live ? min(kc0 + p.cps, p.n_kc) : kc0;
+    const int kc_cta0 = crank * p.ks_cta * p.cps;                        // first chunk of this CTA's K range
+    const int k_cta0 = kc_cta0 * CHUNK_K;
+    const int k_cta1 = min((kc_cta0 + p.ks_cta * p.cps) * CHUNK_K, p.n_kc * CHUNK_K);
+
+    const uint8_t* wptr = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + (rb & 7) * 512 + lane * 16;
+    const uint8_t* sptr = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + kWeightBlockBytes + (rb & 7) * 64 + g * 8;
+
+    auto load_batch = [&](GemvBatch<GROUPED>& b, int kc) {
+#pragma unroll
+        for (int u = 0; u < kGemvUnroll; ++u)
+            if (kc + u < kc1) {
+                b.w[u] = ldg_stream_v4(wptr + (int64_t)u * p.block_bytes);
+                if (GROUPED) b.s[u] = ldg_stream_v2(sptr + (int64_t)u * p.block_bytes);
+            }
+        wptr += (int64_t)kGemvUnroll * p.block_bytes;
+        sptr += (int64_t)kGemvUnroll * p.block_bytes;
+    };
+
+    // Weights do not depend on the previous kernel: start streaming before waiting for it.
+    GemvBatch<GROUPED> cur;
+    load_batch(cur, kc0);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // Stage this CTA's K range of x (zero beyond K) in shared memory.
+    {
+        const int span = k_cta1 - k_cta0;                                // multiple of 32
+        const int vec_per_tok = span >> 3;
+        for (int i = threadIdx.x; i < p.M * vec_per_tok; i += kGemvThreads) {
+            const int m = i / vec_per_tok, v = i - m * vec_per_tok;
+            const int k = k_cta0 + v * 8;
+            uint4 val = make_uint4(0, 0, 0, 0);
+            if (k < p.K) val = *reinterpret_cast<const uint4*>(p.x + (int64_t)m * p.K + k);
+            *reinterpret_cast<uint4*>(xs + m * p.x_stride + v * 8) = val;
+        }
+    }
+    __syncthreads();
+
+    float total[4] = {0.f, 0.f, 0.f, 0.f};
+    const bool tok_live = g < p.M;                                       // this lane supplies token column g
+    const __half* xrow = xs + g * p.x_stride + 8 * c - k_cta0;
+
+    for (int kc = kc0; kc < kc1; kc += kGemvUnroll) {
+        GemvBatch<GROUPED> nxt;
+        if (kc + kGemvUnroll < kc1) load_batch(nxt, kc + kGemvUnroll);
+#pragma unroll
+        for (int u = 0; u < kGemvUnroll; ++u) {
+            if (kc + u < kc1) {
+                const uint4 w = cur.w[u];
+                const __half* xk = xrow + (kc + u) * CHUNK_K;
+                uint32_t a[4];
+                if (BITS == 4) {
+                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint4 xv = make_uint4(0, 0, 0, 0);
+                        if (tok_live) xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
+                        if (GROUPED) {
+                            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                            unpack_int4_word(ww[2 * h], a);
+                            mma_16816(acc, a, xv.x, xv.y);
+                            unpack_int4_word(ww[2 * h + 1], a);
+                            mma_16816(acc, a, xv.z, xv.w);
+                            const uint2 sc = cur.s[u];
+                            const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);   // row g:   G0, G1
+                            const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);   // row g+8: G0, G1
+                            const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
+                            const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
+                            total[0] = fmaf(sg, acc[0], total[0]);
+                            total[1] = fmaf(sg, acc[1], total[1]);
+                            total[2] = fmaf(sg8, acc[2], total[2]);
+                            total[3] = fmaf(sg8, acc[3], total[3]);
+                        } else {
+                            unpack_int4_word(ww[2 * h], a);
+                            mma_16816(total, a, xv.x, xv.y);
+                            unpack_int4_word(ww[2 * h + 1], a);
+                            mma_16816(total, a, xv.z, xv.w);
+                        }
+                    }
+                } else {
+                    uint4 xv = make_uint4(0, 0, 0, 0);
+                    if (tok_live) xv = *reinterpret_cast<const uint4*>(xk);
+                    unpack_int8_words(w.x, w.y, a);
+                    mma_16816(total, a, xv.x, xv.y);
+                    unpack_int8_words(w.z, w.w, a);
+                    mma_16816(total, a, xv.z, xv.w);
+                }
+            }
+        }
+        cur = nxt;
+    }
+
+    // ---- K reduction across warps (shared memory), then across the cluster (distributed shared memory)
+    *reinterpret_cast<float4*>(&red[warp][lane * 4]) = make_float4(total[0], total[1], total[2], total[3]);
+    __syncthreads();
+
+    auto store_out = [&](int rbl, int e, float v) {
+        const int out_rb = rb_group * rb_per_cta + rbl;
+        const int el = e >> 2, i = e & 3;                                // lane that produced it, register index
+        const int row = out_rb * kRbRows + (el >> 2) + 8 * (i >> 1);
+        const int tok = 2 * (el & 3) + (i & 1);
+        if (row < p.N && tok < p.M) {
+            if (!GROUPED) v *= __half2float(p.chan_scales[row]);
+            p.y[(int64_t)tok * p.N + row] = __float2half_rn(v);
+        }
+    };
+
+    const int t = threadIdx.x;
+    if (p.cl > 1) {                                                      // ks_cta == 8: one row-block per CTA
+        cg::cluster_group cluster = cg::this_cluster();
+        if (t < 128) {
+            float v = 0.f;
+            for (int s = 0; s < kGemvWarps; ++s) v += red[s][t];
+            part[t] = v;
+        }
+        cluster.sync();
+        if (crank == 0 && t < 128) {
+            float v = 0.f;
+            for (int r = 0; r < p.cl; ++r) v += *cluster.map_shared_rank(&part[t], r);
+            store_out(0, t, v);
+        }
+        cluster.sync();                                                  // peers keep `part` alive until read
+    } else {
+        for (int idx = t; idx < rb_per_cta * 128; idx += kGemvThreads) {
+            const int rbl = idx >> 7, e = idx & 127;
+            float v = 0.f;
+            for (int s = 0; s < p.ks_cta; ++s) v += red[rbl * p.ks_cta + s][e];
+            store_out(rbl, e, v);
+        }
+    }
+}
+
+}  // namespace ql

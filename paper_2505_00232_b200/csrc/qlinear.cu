@@ -1,0 +1,284 @@
+// C-ABI of the qlinear library: handle life cycle, stage-aware dispatch (paper Section 3.7) and the
+// launchers of the decode and prefill kernels.  Single translation unit for all device code.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/qlinear.h"
+#include "layout.h"
+
+namespace ql {
+// Set by a kernel that gave up a bounded wait: [0] = non-zero code identifying the wait, [1] = count.
+__device__ unsigned int g_device_flag[2];
+}  // namespace ql
+
+#include "dequant.cuh"
+#include "gemv.cuh"
+#include "gemm.cuh"
+
+using namespace ql;
+
+struct GemvPlan {
+    int32_t ks_cta, cl, cps, x_stride, smem_bytes, grid;
+};
+
+struct qlinear_s {
+    Layout L;
+    const uint8_t* blob;
+    int device;
+    int num_sms;
+    int gemv_max_m;
+    bool pdl;
+    GemvPlan gemv[9];          // index = M (1..8)
+    GemmPlan gemm;
+};
+
+namespace {
+
+constexpr int kGemvMaxSmem = 96 * 1024;
+
+int env_int(const char* name, int dflt)
+{
+    const char* v = std::getenv(name);
+    return (v && *v) ? std::atoi(v) : dflt;
+}
+
+GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
+{
+    const int n_rb = (L.N + kRbRows - 1) / kRbRows;
+    const double target = (double)num_sms * env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
+    const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
+    GemvPlan best{};
+    double best_score = -1e30;
+    for (int ks_cta = 1; ks_cta <= 8; ks_cta *= 2)
+        for (int cl = 1; cl <= (ks_cta == 8 ? 8 : 1); ++cl) {
+            const int ks = ks_cta * cl;
+            const int cps = (L.n_kc + ks - 1) / ks;
+            if ((ks - 1) * cps >= L.n_kc && ks > 1) continue;               // would leave a slice empty
+            const int span = std::min(ks_cta * cps, L.n_kc) * L.chunk_k;
+            const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
+            const int smem = M * x_stride * 2;
+            if (smem > kGemvMaxSmem) continue;
+            const double warps = (double)n_rb * ks;
+            const double eff = (double)L.n_kc / ((double)ks * cps);
+            double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 2 ? 1.0 : 0.0);
+            if (force_ks) score = (ks == force_ks) ? 0.0 : -1e29;
+            if (score > best_score) {
+                best_score = score;
+                const int rb_per_cta = kGemvWarps / ks_cta;
+                best = GemvPlan{ks_cta, cl, cps, x_stride, smem, ((n_rb + rb_per_cta - 1) / rb_per_cta) * cl};
+            }
+        }
+    return best;
+}
+
+template <typename Kern, typename Params>
+cudaError_t launch(Kern kern, const Params& prm, dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster, bool pdl)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attrs[2];
+    int na = 0;
+    if (cluster > 1) {
+        attrs[na].id = cudaLaunchAttributeClusterDimension;
+        attrs[na].val.clusterDim.x = cluster;
+        attrs[na].val.clusterDim.y = 1;
+        attrs[na].val.clusterDim.z = 1;
+        ++na;
+    }
+    if (pdl) {
+        attrs[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = na;
+    return cudaLaunchKernelEx(&cfg, kern, prm);
+}
+
+template <int BITS, bool GROUPED>
+cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
+{
+    static bool attr_set[64] = {};
+    auto kern = gemv_kernel<BITS, GROUPED>;
+    if (h->device >= 0 && h->device < 64 && !attr_set[h->device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvMaxSmem);
+        if (e != cudaSuccess) return e;
+        attr_set[h->device] = true;
+    }
+    return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
+}
+
+ql_status forward_gemv(qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
+{
+    const Layout& L = h->L;
+    const GemvPlan& pl = h->gemv[M];
+    GemvParams prm{};
+    prm.body = h->blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
+    prm.x = static_cast<const __half*>(x);
+    prm.y = static_cast<__half*>(y);
+    prm.M = M; prm.N = L.N; prm.K = L.K;
+    prm.n_rb = (L.N + kRbRows - 1) / kRbRows;
+    prm.n_kc = L.n_kc;
+    prm.block_bytes = L.block_bytes;
+    prm.ks_cta = pl.ks_cta; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride;
+    cudaError_t e;
+    if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st);
+    else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st);
+    else e = launch_gemv<4, false>(h, prm, pl, st);
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+// ---- debug: the integers as the device unpack routines see them
+template <int BITS>
+__global__ void __launch_bounds__(256) debug_unpack_kernel(const uint8_t* body, int8_t* q_out, int N, int K,
+                                                           int n_kc, int block_bytes)
+{
+    const int rsb = blockIdx.y, kc = blockIdx.x;
+    const int rb = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+    const uint8_t* blk = body + ((int64_t)rsb * n_kc + kc) * block_bytes;
+    const uint4 w = *reinterpret_cast<const uint4*>(blk + rb * 512 + lane * 16);
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    const int row0 = rsb * kRsbRows + rb * kRbRows + g;
+    constexpr int NMMA = BITS == 4 ? 4 : 2;
+#pragma unroll
+    for (int i = 0; i < NMMA; ++i) {
+        uint32_t a[4];
+        if (BITS == 4) unpack_int4_word(ww[i], a);
+        else unpack_int8_words(ww[2 * i], ww[2 * i + 1], a);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const __half2 hv = *reinterpret_cast<const __half2*>(&a[r]);
+            const int row = row0 + 8 * (r & 1);
+            const int j = 2 * (r >> 1);
+            const int kbase = BITS == 4 ? kc * 64 + int4_k_in_chunk(c, i, j) : kc * 32 + 8 * c + 4 * i + j;
+            if (row < N && kbase < K) {
+                q_out[(int64_t)row * K + kbase] = (int8_t)__half2int_rn(__low2half(hv));
+                q_out[(int64_t)row * K + kbase + 1] = (int8_t)__half2int_rn(__high2half(hv));
+            }
+        }
+    }
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_dev, int device, qlinear_t* out)
+{
+    if (!d || !packed_dev || !out) return QL_ERR_INVALID_ARG;
+    *out = nullptr;
+    Layout L;
+    if (!make_layout(d->N, d->K, d->bits, d->group, &L)) return QL_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(packed_dev) % 256) return QL_ERR_INVALID_ARG;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
+    if (device < 0 || device >= n_dev) return QL_ERR_INVALID_ARG;
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        return QL_ERR_CUDA;
+    if (major != 10) return QL_ERR_ARCH;
+    qlinear_s* h = new (std::nothrow) qlinear_s();
+    if (!h) return QL_ERR_ALLOC;
+    h->L = L;
+    h->blob = static_cast<const uint8_t*>(packed_dev);
+    h->device = device;
+    h->num_sms = sms;
+    h->gemv_max_m = std::max(1, std::min(8, env_int("QLINEAR_GEMV_MAX_M", 8)));
+    h->pdl = env_int("QLINEAR_PDL", 1) != 0;
+    for (int M = 1; M <= 8; ++M) h->gemv[M] = plan_gemv(L, M, sms);
+    ql_status st = gemm_plan(L, sms, &h->gemm);
+    if (st != QL_OK) { delete h; return st; }
+    *out = h;
+    return QL_OK;
+}
+
+extern "C" int32_t qlinear_path_for(qlinear_t h, int32_t M)
+{
+    if (!h || M < 1) return 0;
+    return M <= h->gemv_max_m ? QL_PATH_GEMV : QL_PATH_GEMM;
+}
+
+extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_t M, void* stream)
+{
+    if (!h || !x || !y || M < 1) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
+    if ((int64_t)M * h->L.K > INT32_MAX || (int64_t)M * h->L.N > INT32_MAX) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (M <= h->gemv_max_m) return forward_gemv(h, x, y, M, st);
+    return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl);
+}
+
+extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, void* stream)
+{
+    if (!h || !q_out) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    const Layout& L = h->L;
+    dim3 grid(L.n_kc, L.n_rsb);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (L.bits == 4)
+        debug_unpack_kernel<4><<<grid, 256, 0, st>>>(h->blob + L.body_offset, q_out, L.N, L.K, L.n_kc, L.block_bytes);
+    else
+        debug_unpack_kernel<8><<<grid, 256, 0, st>>>(h->blob + L.body_offset, q_out, L.N, L.K, L.n_kc, L.block_bytes);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_device_status(qlinear_t h, uint32_t* detail)
+{
+    if (!h) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    unsigned int flag[2] = {0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
+    if (cudaMemcpyFromSymbol(flag, g_device_flag, sizeof(flag)) != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
+    if (detail) *detail = flag[0];
+    if (flag[0] == 0) return QL_OK;
+    const unsigned int zero[2] = {0, 0};
+    cudaMemcpyToSymbol(g_device_flag, zero, sizeof(zero));
+    return QL_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" ql_status qlinear_destroy(qlinear_t h)
+{
+    delete h;
+    return QL_OK;
+}
+
+extern "C" const char* qlinear_status_string(ql_status s)
+{
+    switch (s) {
+        case QL_OK: return "ok";
+        case QL_ERR_INVALID_ARG: return "invalid argument";
+        case QL_ERR_UNSUPPORTED: return "unsupported shape or quantisation scheme";
+        case QL_ERR_ALLOC: return "host allocation failed";
+        case QL_ERR_CUDA: return "CUDA call failed";
+        case QL_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case QL_ERR_ARCH: return "device is not compute capability 10.x (sm_100)";
+    }
+    return "unknown status";
+}
+
+extern "C" uint32_t qlinear_version(void) { return (1u << 16) | 0u; }

@@ -17,3 +17,22 @@ def golden():
     import json
     with open(os.path.join(ROOT, "tests", "golden", "worked_examples.json")) as f:
         return json.load(f)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_library():
+    """The C-ABI library is built in-tree (nvcc cross-compiles without a GPU); rebuild if stale."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_qlinear_build", os.path.join(ROOT, "paper_2505_00232_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    mod.build()
+    yield
+
+
+def has_gpu() -> bool:
+    try:
+        import torch
+        return torch.cuda.is_available()
+    except Exception:
+        return False
