@@ -228,7 +228,7 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (M <= h->gemv_max_m) return forward_gemv(h, x, y, M, st);
-    return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl);
+    return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
 extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, void* stream)
