@@ -308,6 +308,8 @@ def main():
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill sub-measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill-steps", type=int, default=20)
+    ap.add_argument("--quick", action="store_true",
+                    help="main timed region only (no e2e, per-kernel, prefill or CPU legs): the command to profile")
     args = ap.parse_args()
 
     workload = C.by_name(args.workload)
@@ -352,6 +354,16 @@ def main():
     steps = res["steps"]
     units_per_step = units_of(stage, ls.weight_bytes, ls.flops)
     value = world * units_per_step * steps / (res["ms"] / 1e3)
+
+    if args.quick:
+        if rank == 0:
+            print(json.dumps({"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": steps,
+                              "warmup": args.warmup, "ms_per_step": res["ms"] / steps, "quick": True,
+                              "config": {"workload": workload.name, "M": M, "weight_copies": copies},
+                              "gpu_launches": res["launches"]}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end through the public API with host buffers (H2D + forwards + D2H per step)
     e2e_steps = max(8, min(200, steps // 10))

@@ -26,7 +26,7 @@ namespace cg = cooperative_groups;
 
 constexpr int kGemvWarps = 8;
 constexpr int kGemvThreads = kGemvWarps * 32;
-constexpr int kGemvUnroll = 4;           // chunks in flight per lane per batch
+constexpr int kGemvRing = 8;             // chunks prefetched per warp (cp.async ring slots)
 
 struct GemvParams {
     const uint8_t* body;                 // first block of the packed body
@@ -41,6 +41,7 @@ struct GemvParams {
     int32_t cl;                          // CTAs per cluster along K (1 = no cluster)
     int32_t cps;                         // chunks per slice
     int32_t x_stride;                    // halves between tokens in the shared x slab
+    int32_t x_bytes;                     // bytes of the x slab (the warp rings follow it)
 };
 
 __device__ __forceinline__ uint4 ldg_stream_v4(const void* p)
@@ -65,14 +66,16 @@ __device__ __forceinline__ void mma_16816(float d[4], const uint32_t a[4], uint3
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <bool GROUPED>
-struct GemvBatch {
-    uint4 w[kGemvUnroll];
-    uint2 s[GROUPED ? kGemvUnroll : 1];
-};
+// Same instruction without `volatile`: the compiler may interleave independent MMA chains.
+__device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
 template <int BITS, bool GROUPED>
-__global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const GemvParams p)
+__global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __half* xs = reinterpret_cast<__half*>(smem_raw);                   // [M][x_stride]
@@ -96,23 +99,31 @@ __global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const GemvParams p)
     const int k_cta0 = kc_cta0 * CHUNK_K;
     const int k_cta1 = min((kc_cta0 + p.ks_cta * p.cps) * CHUNK_K, p.n_kc * CHUNK_K);
 
-    const uint8_t* wptr = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + (rb & 7) * 512 + lane * 16;
-    const uint8_t* sptr = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + kWeightBlockBytes + (rb & 7) * 64 + g * 8;
+    // Warp-private ring of kGemvRing chunk slots filled by cp.async: the prefetch depth does not cost
+    // registers, and a lane reads back exactly the 16 bytes it copied (the 64 bytes of group scales are
+    // copied by lanes 0..3 and shared through __syncwarp).
+    constexpr int SLOT = GROUPED ? 576 : 512;
+    unsigned char* ring = smem_raw + p.x_bytes + warp * (kGemvRing * SLOT);
+    const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ring);
+    const uint8_t* blk = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + (rb & 7) * 512;
+    const uint8_t* wsrc = blk + lane * 16;
+    const uint8_t* ssrc = blk + kWeightBlockBytes - (rb & 7) * 512 + (rb & 7) * 64 + (lane & 3) * 16;
 
-    auto load_batch = [&](GemvBatch<GROUPED>& b, int kc) {
-#pragma unroll
-        for (int u = 0; u < kGemvUnroll; ++u)
-            if (kc + u < kc1) {
-                b.w[u] = ldg_stream_v4(wptr + (int64_t)u * p.block_bytes);
-                if (GROUPED) b.s[u] = ldg_stream_v2(sptr + (int64_t)u * p.block_bytes);
-            }
-        wptr += (int64_t)kGemvUnroll * p.block_bytes;
-        sptr += (int64_t)kGemvUnroll * p.block_bytes;
+    auto issue = [&](int kc, int slot) {                                 // always commits, so group counts stay uniform
+        if (kc < kc1) {
+            const uint32_t dst = ring_u32 + slot * SLOT;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + lane * 16), "l"(wsrc) : "memory");
+            if (GROUPED && lane < 4)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 512 + lane * 16), "l"(ssrc) : "memory");
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        wsrc += p.block_bytes;
+        ssrc += p.block_bytes;
     };
 
-    // Weights do not depend on the previous kernel: start streaming before waiting for it.
-    GemvBatch<GROUPED> cur;
-    load_batch(cur, kc0);
+    // Weights do not depend on the previous kernel: fill the ring before waiting for it.
+#pragma unroll
+    for (int d = 0; d < kGemvRing; ++d) issue(kc0 + d, d);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -131,58 +142,61 @@ __global__ void __launch_bounds__(kGemvThreads) gemv_kernel(const GemvParams p)
     __syncthreads();
 
     float total[4] = {0.f, 0.f, 0.f, 0.f};
-    const bool tok_live = g < p.M;                                       // this lane supplies token column g
-    const __half* xrow = xs + g * p.x_stride + 8 * c - k_cta0;
+    // Lanes whose token column does not exist (g >= M) read the last real token: MMA columns are
+    // independent and those columns are never stored.
+    const __half* xrow = xs + min(g, p.M - 1) * p.x_stride + 8 * c - k_cta0;
 
-    for (int kc = kc0; kc < kc1; kc += kGemvUnroll) {
-        GemvBatch<GROUPED> nxt;
-        if (kc + kGemvUnroll < kc1) load_batch(nxt, kc + kGemvUnroll);
+    int slot = 0;
+    for (int kc = kc0; kc < kc1; ++kc) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 1) : "memory");
+        if (GROUPED) __syncwarp();
+        const unsigned char* sp = ring + slot * SLOT;
+        const uint4 w = *reinterpret_cast<const uint4*>(sp + lane * 16);
+        uint2 sc = make_uint2(0, 0);
+        if (GROUPED) {
+            sc = *reinterpret_cast<const uint2*>(sp + 512 + g * 8);
+            __syncwarp();                                                // every lane has its scales before the refill
+        }
+        issue(kc + kGemvRing, slot);
+        slot = slot + 1 == kGemvRing ? 0 : slot + 1;
+
+        const __half* xk = xrow + kc * CHUNK_K;
+        uint32_t a[4];
+        if (BITS == 4) {
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-        for (int u = 0; u < kGemvUnroll; ++u) {
-            if (kc + u < kc1) {
-                const uint4 w = cur.w[u];
-                const __half* xk = xrow + (kc + u) * CHUNK_K;
-                uint32_t a[4];
-                if (BITS == 4) {
-                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint4 xv = make_uint4(0, 0, 0, 0);
-                        if (tok_live) xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
-                        if (GROUPED) {
-                            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                            unpack_int4_word(ww[2 * h], a);
-                            mma_16816(acc, a, xv.x, xv.y);
-                            unpack_int4_word(ww[2 * h + 1], a);
-                            mma_16816(acc, a, xv.z, xv.w);
-                            const uint2 sc = cur.s[u];
-                            const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);   // row g:   G0, G1
-                            const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);   // row g+8: G0, G1
-                            const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
-                            const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
-                            total[0] = fmaf(sg, acc[0], total[0]);
-                            total[1] = fmaf(sg, acc[1], total[1]);
-                            total[2] = fmaf(sg8, acc[2], total[2]);
-                            total[3] = fmaf(sg8, acc[3], total[3]);
-                        } else {
-                            unpack_int4_word(ww[2 * h], a);
-                            mma_16816(total, a, xv.x, xv.y);
-                            unpack_int4_word(ww[2 * h + 1], a);
-                            mma_16816(total, a, xv.z, xv.w);
-                        }
-                    }
+            for (int h = 0; h < 2; ++h) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
+                if (GROUPED) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    unpack_int4_word(ww[2 * h], a);
+                    mma_16816_pure(acc, a, xv.x, xv.y);
+                    unpack_int4_word(ww[2 * h + 1], a);
+                    mma_16816_pure(acc, a, xv.z, xv.w);
+                    const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);          // row g:   G0, G1
+                    const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);          // row g+8: G0, G1
+                    const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
+                    const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
+                    total[0] = fmaf(sg, acc[0], total[0]);
+                    total[1] = fmaf(sg, acc[1], total[1]);
+                    total[2] = fmaf(sg8, acc[2], total[2]);
+                    total[3] = fmaf(sg8, acc[3], total[3]);
                 } else {
-                    uint4 xv = make_uint4(0, 0, 0, 0);
-                    if (tok_live) xv = *reinterpret_cast<const uint4*>(xk);
-                    unpack_int8_words(w.x, w.y, a);
-                    mma_16816(total, a, xv.x, xv.y);
-                    unpack_int8_words(w.z, w.w, a);
-                    mma_16816(total, a, xv.z, xv.w);
+                    unpack_int4_word(ww[2 * h], a);
+                    mma_16816_pure(total, a, xv.x, xv.y);
+                    unpack_int4_word(ww[2 * h + 1], a);
+                    mma_16816_pure(total, a, xv.z, xv.w);
                 }
             }
+        } else {
+            const uint4 xv = *reinterpret_cast<const uint4*>(xk);
+            unpack_int8_words(w.x, w.y, a);
+            mma_16816_pure(total, a, xv.x, xv.y);
+            unpack_int8_words(w.z, w.w, a);
+            mma_16816_pure(total, a, xv.z, xv.w);
         }
-        cur = nxt;
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 
     // ---- K reduction across warps (shared memory), then across the cluster (distributed shared memory)
     *reinterpret_cast<float4*>(&red[warp][lane * 4]) = make_float4(total[0], total[1], total[2], total[3]);

@@ -19,12 +19,13 @@ __device__ unsigned int g_device_flag[2];
 
 #include "dequant.cuh"
 #include "gemv.cuh"
+#include "gemv_stream.cuh"
 #include "gemm.cuh"
 
 using namespace ql;
 
 struct GemvPlan {
-    int32_t ks_cta, cl, cps, x_stride, smem_bytes, grid;
+    int32_t ks_cta, cl, cps, x_stride, x_bytes, smem_bytes, grid;
 };
 
 struct qlinear_s {
@@ -36,6 +37,11 @@ struct qlinear_s {
     bool pdl;
     GemvPlan gemv[9];          // index = M (1..8)
     GemmPlan gemm;
+    // streaming decode kernel
+    int gemv_kernel_choice;    // 0 = cluster kernel, 1 = streaming kernel
+    int stream_P, stream_stages;
+    float* stream_scratch;     // device, owned: [P][2][1024] fp32 partial sums
+    unsigned int* stream_counters;   // device, owned: [n_rsb][8], zero between launches
 };
 
 namespace {
@@ -62,7 +68,8 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             if ((ks - 1) * cps >= L.n_kc && ks > 1) continue;               // would leave a slice empty
             const int span = std::min(ks_cta * cps, L.n_kc) * L.chunk_k;
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
-            const int smem = M * x_stride * 2;
+            const int x_bytes = ((M * x_stride * 2 + 127) / 128) * 128;
+            const int smem = x_bytes + kGemvWarps * kGemvRing * (L.grouped ? 576 : 512);
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
             const double eff = (double)L.n_kc / ((double)ks * cps);
@@ -71,7 +78,7 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             if (score > best_score) {
                 best_score = score;
                 const int rb_per_cta = kGemvWarps / ks_cta;
-                best = GemvPlan{ks_cta, cl, cps, x_stride, smem, ((n_rb + rb_per_cta - 1) / rb_per_cta) * cl};
+                best = GemvPlan{ks_cta, cl, cps, x_stride, x_bytes, smem, ((n_rb + rb_per_cta - 1) / rb_per_cta) * cl};
             }
         }
     return best;
@@ -130,11 +137,61 @@ ql_status forward_gemv(qlinear_s* h, const void* x, void* y, int M, cudaStream_t
     prm.n_rb = (L.N + kRbRows - 1) / kRbRows;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
-    prm.ks_cta = pl.ks_cta; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride;
+    prm.ks_cta = pl.ks_cta; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
     cudaError_t e;
     if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st);
     else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st);
     else e = launch_gemv<4, false>(h, prm, pl, st);
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+template <int BITS, bool GROUPED, int NS>
+cudaError_t launch_stream_ns(const qlinear_s* h, const StreamParams& prm, cudaStream_t st)
+{
+    static bool attr_set[64] = {};
+    auto kern = gemv_stream_kernel<BITS, GROUPED, NS>;
+    if (h->device >= 0 && h->device < 64 && !attr_set[h->device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, NS * StreamStage<BITS>::kBytes);
+        if (e != cudaSuccess) return e;
+        attr_set[h->device] = true;
+    }
+    return launch(kern, prm, dim3(prm.P), dim3(kStreamThreads), (size_t)NS * StreamStage<BITS>::kBytes, st, 1, h->pdl);
+}
+
+template <int BITS, bool GROUPED>
+cudaError_t launch_stream(const qlinear_s* h, const StreamParams& prm, cudaStream_t st)
+{
+    switch (prm.stages) {
+        case 6: return launch_stream_ns<BITS, GROUPED, 6>(h, prm, st);
+        case 8: return launch_stream_ns<BITS, GROUPED, 8>(h, prm, st);
+        case 12: return launch_stream_ns<BITS, GROUPED, 12>(h, prm, st);
+        case 16: return launch_stream_ns<BITS, GROUPED, 16>(h, prm, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+ql_status forward_gemv_stream(qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
+{
+    const Layout& L = h->L;
+    StreamParams prm{};
+    prm.body = h->blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
+    prm.x = static_cast<const __half*>(x);
+    prm.y = static_cast<__half*>(y);
+    prm.scratch = h->stream_scratch;
+    prm.counters = h->stream_counters;
+    prm.M = M; prm.N = L.N; prm.K = L.K;
+    prm.n_rsb = L.n_rsb; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
+    prm.P = h->stream_P;
+    prm.stages = h->stream_stages;
+#ifdef QL_TRACE
+    static int trace_seq = 0;
+    prm.trace_seq = trace_seq++;
+#endif
+    cudaError_t e;
+    if (L.bits == 8) e = launch_stream<8, false>(h, prm, st);
+    else if (L.grouped) e = launch_stream<4, true>(h, prm, st);
+    else e = launch_stream<4, false>(h, prm, st);
     return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
@@ -209,6 +266,27 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
     for (int M = 1; M <= 8; ++M) h->gemv[M] = plan_gemv(L, M, sms);
     ql_status st = gemm_plan(L, sms, &h->gemm);
     if (st != QL_OK) { delete h; return st; }
+    // streaming decode kernel: persistent grid, ring depth and per-handle scratch
+    {
+        const int stage_bytes = L.bits == 4 ? StreamStage<4>::kBytes : StreamStage<8>::kBytes;
+        const int ctas_per_sm = std::max(1, std::min(4, env_int("QLINEAR_STREAM_CTAS_PER_SM", 3)));
+        const int max_stages = std::min(env_int("QLINEAR_STREAM_STAGES", kStreamMaxStages), (220 * 1024 / ctas_per_sm - 1536) / stage_bytes);
+        h->stream_stages = max_stages >= 16 ? 16 : max_stages >= 12 ? 12 : max_stages >= 8 ? 8 : 6;   // instantiated ring depths
+        const int64_t B = (int64_t)L.n_rsb * L.n_kc;
+        h->stream_P = (int)std::min<int64_t>(B, (int64_t)sms * ctas_per_sm);
+        const char* kc = std::getenv("QLINEAR_GEMV_KERNEL");
+        const int64_t body_bytes = B * L.block_bytes;
+        h->gemv_kernel_choice = (kc && !std::strcmp(kc, "cluster")) ? 0 : (kc && !std::strcmp(kc, "stream")) ? 1
+                                : (body_bytes >= env_int("QLINEAR_STREAM_MIN_BYTES", 1 << 20) ? 1 : 0);
+        if (L.bits == 4 && (L.K % 64)) h->gemv_kernel_choice = 0;       // the streaming kernel reads whole 64-k slices of x
+        DeviceGuard guard(device);
+        const size_t sbytes = (size_t)h->stream_P * 2 * kStreamPartialFloats * sizeof(float);
+        const size_t cbytes = (size_t)L.n_rsb * 8 * sizeof(unsigned int);
+        if (!guard.ok || cudaMalloc(&h->stream_scratch, sbytes) != cudaSuccess) { cudaGetLastError(); delete h; return QL_ERR_CUDA; }
+        if (cudaMalloc(&h->stream_counters, cbytes) != cudaSuccess || cudaMemset(h->stream_counters, 0, cbytes) != cudaSuccess) {
+            cudaGetLastError(); cudaFree(h->stream_scratch); cudaFree(h->stream_counters); delete h; return QL_ERR_CUDA;
+        }
+    }
     *out = h;
     return QL_OK;
 }
@@ -227,7 +305,7 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (M <= h->gemv_max_m) return forward_gemv(h, x, y, M, st);
+    if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(h, x, y, M, st);
     return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
@@ -263,6 +341,12 @@ extern "C" ql_status qlinear_device_status(qlinear_t h, uint32_t* detail)
 
 extern "C" ql_status qlinear_destroy(qlinear_t h)
 {
+    if (!h) return QL_OK;
+    {
+        DeviceGuard guard(h->device);
+        cudaFree(h->stream_scratch);
+        cudaFree(h->stream_counters);
+    }
     delete h;
     return QL_OK;
 }
@@ -280,5 +364,12 @@ extern "C" const char* qlinear_status_string(ql_status s)
     }
     return "unknown status";
 }
+
+#ifdef QL_TRACE
+extern "C" int qlinear_debug_read_trace(unsigned long long* out, size_t bytes)
+{
+    return (int)cudaMemcpyFromSymbol(out, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
+}
+#endif
 
 extern "C" uint32_t qlinear_version(void) { return (1u << 16) | 0u; }
