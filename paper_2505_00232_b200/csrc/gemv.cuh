@@ -44,21 +44,6 @@ struct GemvParams {
     int32_t x_bytes;                     // bytes of the x slab (the warp rings follow it)
 };
 
-__device__ __forceinline__ uint4 ldg_stream_v4(const void* p)
-{
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
-__device__ __forceinline__ uint2 ldg_stream_v2(const void* p)
-{
-    uint2 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-    return v;
-}
-
 __device__ __forceinline__ void mma_16816(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
 {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -100,30 +85,35 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     const int k_cta1 = min((kc_cta0 + p.ks_cta * p.cps) * CHUNK_K, p.n_kc * CHUNK_K);
 
     // Warp-private ring of kGemvRing chunk slots filled by cp.async: the prefetch depth does not cost
-    // registers, and a lane reads back exactly the 16 bytes it copied (the 64 bytes of group scales are
-    // copied by lanes 0..3 and shared through __syncwarp).
-    constexpr int SLOT = GROUPED ? 576 : 512;
-    unsigned char* ring = smem_raw + p.x_bytes + warp * (kGemvRing * SLOT);
-    const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ring);
-    const uint8_t* blk = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes + (rb & 7) * 512;
-    const uint8_t* wsrc = blk + lane * 16;
-    const uint8_t* ssrc = blk + kWeightBlockBytes - (rb & 7) * 512 + (rb & 7) * 64 + (lane & 3) * 16;
+    // registers and a lane reads back exactly the 16 bytes it copied.  The group scales of a whole
+    // ring pass (8 chunks x 64 bytes) are fetched by one extra 16-byte copy per lane into one of two
+    // per-warp pass buffers.  The steady state has no divergent branch.
+    static_assert(kGemvRing == 8, "one scale copy per lane covers exactly 8 chunks");
+    constexpr int WARP_SMEM = kGemvRing * 512 + (GROUPED ? 2 * 512 : 0);
+    unsigned char* ring = smem_raw + p.x_bytes + warp * WARP_SMEM;
+    unsigned char* sbuf = ring + kGemvRing * 512;
+    const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ring) + lane * 16;
+    const uint32_t sbuf_u32 = (uint32_t)__cvta_generic_to_shared(sbuf) + lane * 16;
+    const uint8_t* blk = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes;
+    const uint8_t* wsrc = blk + (rb & 7) * 512 + lane * 16;
+    // lane L copies part (L & 3) of the scales of chunk (pass start + L / 4)
+    const uint8_t* ssrc = blk + (int64_t)(lane >> 2) * p.block_bytes + kWeightBlockBytes + (rb & 7) * 64 + (lane & 3) * 16;
+    const int64_t pass_bytes = (int64_t)kGemvRing * p.block_bytes;
 
-    auto issue = [&](int kc, int slot) {                                 // always commits, so group counts stay uniform
-        if (kc < kc1) {
-            const uint32_t dst = ring_u32 + slot * SLOT;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + lane * 16), "l"(wsrc) : "memory");
-            if (GROUPED && lane < 4)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 512 + lane * 16), "l"(ssrc) : "memory");
-        }
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        wsrc += p.block_bytes;
-        ssrc += p.block_bytes;
+    auto copy16 = [](uint32_t dst, const void* src, bool in_range) {     // out of range: reads nothing, writes zeros
+        const uint32_t sz = in_range ? 16u : 0u;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
     };
+    auto commit = [] { asm volatile("cp.async.commit_group;" ::: "memory"); };
 
     // Weights do not depend on the previous kernel: fill the ring before waiting for it.
+    if (GROUPED) { copy16(sbuf_u32, ssrc, kc0 + (lane >> 2) < kc1); ssrc += pass_bytes; }
 #pragma unroll
-    for (int d = 0; d < kGemvRing; ++d) issue(kc0 + d, d);
+    for (int d = 0; d < kGemvRing; ++d) {
+        copy16(ring_u32 + d * 512, wsrc, kc0 + d < kc1);
+        commit();
+        wsrc += p.block_bytes;
+    }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -144,57 +134,65 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     float total[4] = {0.f, 0.f, 0.f, 0.f};
     // Lanes whose token column does not exist (g >= M) read the last real token: MMA columns are
     // independent and those columns are never stored.
-    const __half* xrow = xs + min(g, p.M - 1) * p.x_stride + 8 * c - k_cta0;
+    const __half* xpass = xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
+    const unsigned char* wslot = ring + lane * 16;
+    int sflip = 0;                                                       // scale buffer of the current pass
 
-    int slot = 0;
-    for (int kc = kc0; kc < kc1; ++kc) {
-        asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 1) : "memory");
-        if (GROUPED) __syncwarp();
-        const unsigned char* sp = ring + slot * SLOT;
-        const uint4 w = *reinterpret_cast<const uint4*>(sp + lane * 16);
-        uint2 sc = make_uint2(0, 0);
-        if (GROUPED) {
-            sc = *reinterpret_cast<const uint2*>(sp + 512 + g * 8);
-            __syncwarp();                                                // every lane has its scales before the refill
-        }
-        issue(kc + kGemvRing, slot);
-        slot = slot + 1 == kGemvRing ? 0 : slot + 1;
-
-        const __half* xk = xrow + kc * CHUNK_K;
-        uint32_t a[4];
-        if (BITS == 4) {
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    for (int kc = kc0; kc < kc1; kc += kGemvRing) {
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
-                if (GROUPED) {
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                    unpack_int4_word(ww[2 * h], a);
-                    mma_16816_pure(acc, a, xv.x, xv.y);
-                    unpack_int4_word(ww[2 * h + 1], a);
-                    mma_16816_pure(acc, a, xv.z, xv.w);
-                    const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);          // row g:   G0, G1
-                    const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);          // row g+8: G0, G1
-                    const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
-                    const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
-                    total[0] = fmaf(sg, acc[0], total[0]);
-                    total[1] = fmaf(sg, acc[1], total[1]);
-                    total[2] = fmaf(sg8, acc[2], total[2]);
-                    total[3] = fmaf(sg8, acc[3], total[3]);
-                } else {
-                    unpack_int4_word(ww[2 * h], a);
-                    mma_16816_pure(total, a, xv.x, xv.y);
-                    unpack_int4_word(ww[2 * h + 1], a);
-                    mma_16816_pure(total, a, xv.z, xv.w);
-                }
+        for (int d = 0; d < kGemvRing; ++d) {
+            if (kc + d >= kc1) break;
+            asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 1) : "memory");
+            if (GROUPED && d == 0) {
+                __syncwarp();                                            // scales of this pass visible; last pass's reads done
+                copy16(sbuf_u32 + (sflip ^ 1) * 512, ssrc, kc + kGemvRing + (lane >> 2) < kc1);
+                ssrc += pass_bytes;
             }
-        } else {
-            const uint4 xv = *reinterpret_cast<const uint4*>(xk);
-            unpack_int8_words(w.x, w.y, a);
-            mma_16816_pure(total, a, xv.x, xv.y);
-            unpack_int8_words(w.z, w.w, a);
-            mma_16816_pure(total, a, xv.z, xv.w);
+            const uint4 w = *reinterpret_cast<const uint4*>(wslot + d * 512);
+            uint2 sc = make_uint2(0, 0);
+            if (GROUPED) sc = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + d * 64 + g * 8);
+            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slot just read
+            commit();
+            wsrc += p.block_bytes;
+
+            const __half* xk = xpass + d * CHUNK_K;
+            uint32_t a[4];
+            if (BITS == 4) {
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint4 xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
+                    if (GROUPED) {
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        unpack_int4_word(ww[2 * h], a);
+                        mma_16816_pure(acc, a, xv.x, xv.y);
+                        unpack_int4_word(ww[2 * h + 1], a);
+                        mma_16816_pure(acc, a, xv.z, xv.w);
+                        const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);      // row g:   G0, G1
+                        const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);      // row g+8: G0, G1
+                        const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
+                        const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
+                        total[0] = fmaf(sg, acc[0], total[0]);
+                        total[1] = fmaf(sg, acc[1], total[1]);
+                        total[2] = fmaf(sg8, acc[2], total[2]);
+                        total[3] = fmaf(sg8, acc[3], total[3]);
+                    } else {
+                        unpack_int4_word(ww[2 * h], a);
+                        mma_16816_pure(total, a, xv.x, xv.y);
+                        unpack_int4_word(ww[2 * h + 1], a);
+                        mma_16816_pure(total, a, xv.z, xv.w);
+                    }
+                }
+            } else {
+                const uint4 xv = *reinterpret_cast<const uint4*>(xk);
+                unpack_int8_words(w.x, w.y, a);
+                mma_16816_pure(total, a, xv.x, xv.y);
+                unpack_int8_words(w.z, w.w, a);
+                mma_16816_pure(total, a, xv.z, xv.w);
+            }
         }
+        xpass += kGemvRing * CHUNK_K;
+        sflip ^= 1;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 

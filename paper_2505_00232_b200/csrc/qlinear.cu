@@ -69,7 +69,7 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             const int span = std::min(ks_cta * cps, L.n_kc) * L.chunk_k;
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
             const int x_bytes = ((M * x_stride * 2 + 127) / 128) * 128;
-            const int smem = x_bytes + kGemvWarps * kGemvRing * (L.grouped ? 576 : 512);
+            const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
             const double eff = (double)L.n_kc / ((double)ks * cps);
@@ -277,7 +277,7 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
         const char* kc = std::getenv("QLINEAR_GEMV_KERNEL");
         const int64_t body_bytes = B * L.block_bytes;
         h->gemv_kernel_choice = (kc && !std::strcmp(kc, "cluster")) ? 0 : (kc && !std::strcmp(kc, "stream")) ? 1
-                                : (body_bytes >= env_int("QLINEAR_STREAM_MIN_BYTES", 1 << 20) ? 1 : 0);
+                                : (body_bytes >= (int64_t)env_int("QLINEAR_STREAM_MIN_MB", 1 << 20) * (1 << 20) ? 1 : 0);
         if (L.bits == 4 && (L.K % 64)) h->gemv_kernel_choice = 0;       // the streaming kernel reads whole 64-k slices of x
         DeviceGuard guard(device);
         const size_t sbytes = (size_t)h->stream_P * 2 * kStreamPartialFloats * sizeof(float);
