@@ -161,6 +161,22 @@ class LayerSet:
         return sum(2 * self.M * l.N for l in self.layers)
 
 
+def max_over_ranks(local_value: float, device) -> float:
+    """Slowest rank's value (all-reduce MAX); identity when no process group is up."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(local_value)
+    t = torch.tensor([local_value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_step: float, steps: int, ms: float, world: int) -> float:
+    """Replicas only: every rank processes the same units; the job's rate uses the slowest rank's time."""
+    return world * units_per_step * steps / (ms / 1e3)
+
+
 def time_events(torch, fn, iters):
     """Device time of fn() repeated `iters` times on the current stream (CUDA events), in ms."""
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -348,12 +364,10 @@ def main():
     res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local))
     if world > 1:
         dist.barrier()
-        t = torch.tensor([res["ms"]], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        res["ms"] = float(t.item())
+        res["ms"] = max_over_ranks(res["ms"], device)
     steps = res["steps"]
     units_per_step = units_of(stage, ls.weight_bytes, ls.flops)
-    value = world * units_per_step * steps / (res["ms"] / 1e3)
+    value = whole_job_value(units_per_step, steps, res["ms"], world)
 
     if args.quick:
         if rank == 0:
@@ -374,11 +388,8 @@ def main():
     for i in range(e2e_steps):
         ls.step_e2e(i % copies)
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * units_per_step * e2e_steps / e2e_s
+    e2e_s = max_over_ranks(e2e_s, device)
+    e2e_value = whole_job_value(units_per_step, e2e_steps, e2e_s * 1e3, world)
 
     # ---- roofline of the dominant kernel (live CUDA-event timing of that kernel's launches alone)
     if stage == "decode":

@@ -158,3 +158,23 @@ def test_parity_decode_configs_full_size(P, torch, w, li, M):
     # device-side integers, sampled rows (full compare for the small layers)
     qd = lin.debug_unpack().cpu().numpy()
     assert (qd == q).all()
+
+
+@pytest.mark.parametrize("M,N,K,bits,group", [(1, 2304, 2304, 8, 0), (3, 264, 2304, 4, 32), (8, 1024, 4096, 4, 32),
+                                              (2, 4096, 4096, 8, 0), (5, 384, 4096, 4, 0), (1, 520, 1056, 8, 0)])
+def test_streaming_kernel_parity(P, torch, monkeypatch, M, N, K, bits, group):
+    """The optional persistent streaming decode kernel (selected at handle creation) meets the same bar."""
+    monkeypatch.setenv("QLINEAR_GEMV_KERNEL", "stream")
+    q, s, x = rand_case(3000 + N + K, M, N, K, bits, group)
+    lin, y = run_layer(P, torch, q, s, bits, group, x)
+    assert_parity(y, x, q, s, group)
+    xd = torch.from_numpy(x).cuda()
+    a = lin.forward(xd).clone()
+    for _ in range(3):
+        assert torch.equal(a, lin.forward(xd))           # counters reset themselves between launches
+    xo = np.zeros_like(x)
+    xo[:, 7] = 1.0
+    G = K if group == 0 else group
+    want = (s[:, 7 // G].astype(np.float64) * q[:, 7].astype(np.float64)).astype(np.float16)
+    yo = lin.forward(torch.from_numpy(xo).cuda()).cpu().numpy()
+    assert (yo.view(np.uint16) == want.view(np.uint16)[None, :]).all()
