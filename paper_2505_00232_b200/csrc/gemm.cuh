@@ -4,15 +4,17 @@
 //
 // The product is computed transposed, D[n, m] = sum_k W[n,k] * x[m,k]: the 128 output channels of a
 // row super-block are the MMA's M dimension, the tokens its N dimension, so that each dequantised
-// weight is reused by up to 256 tokens.  Per CTA:
+// weight is reused by up to 256 tokens.  The grid is persistent (one CTA per SM, tiles assigned
+// round-robin) and the accumulator is double-buffered in tensor memory, so the epilogue of one tile
+// runs under the main loop of the next.  Per CTA:
 //
-//   warp 0       producer: one bulk copy of the packed weight block(s) of the k-step (contiguous in
-//                the blob) and one TMA tile load of x [BN tokens x 64 k] (128-byte swizzle)
-//   warps 2..9   dequantise: packed block (shared) -> registers -> exact fp16 integers (x group scale
-//                for grouped int4) -> the K-major 128-byte-swizzled A tile in shared memory
-//   warp 1       issues tcgen05.mma (A, B from shared memory, fp32 accumulator in tensor memory) and
-//                frees pipeline stages with tcgen05.commit
-//   warps 2..9   epilogue: tcgen05.ld the accumulator, apply the per-channel scale, round to fp16, store
+//   warp 0        producer: one bulk copy of the packed weight block(s) of the k-step (contiguous in
+//                 the blob) and one TMA tile load of x [BN tokens x 64 k] (128-byte swizzle, no multicast)
+//   warps 2..17   dequantise: packed block (shared) -> registers -> exact fp16 integers (x group scale
+//                 for grouped int4) -> the K-major 128-byte-swizzled A tile in shared memory
+//   warp 1        issues tcgen05.mma (A, B from shared memory, fp32 accumulator in tensor memory),
+//                 frees pipeline stages and publishes finished accumulators with tcgen05.commit
+//   warps 18..21  epilogue: tcgen05.ld the accumulator, apply the per-channel scale, round to fp16, store
 //
 // Every mbarrier wait is bounded: on expiry the kernel records a code in g_device_flag, every role
 // leaves its loop, tensor memory is released and the kernel returns.
@@ -29,8 +31,9 @@
 
 namespace ql {
 
-constexpr int kGemmThreads = 320;            // 10 warps
-constexpr int kGemmDequantWarps = 8;
+constexpr int kGemmDequantWarps = 16;
+constexpr int kGemmEpilogueWarps = 4;
+constexpr int kGemmThreads = (2 + kGemmDequantWarps + kGemmEpilogueWarps) * 32;   // 22 warps
 constexpr int kGemmKStep = 64;               // k per pipeline stage = one 128-byte swizzle row of fp16
 constexpr int kGemmATileBytes = 128 * 128;   // 128 rows x 64 fp16
 
@@ -41,16 +44,81 @@ struct GemmParams {
     int32_t M, N, K;
     int32_t n_kc, block_bytes;
     int32_t n_ksteps;
+    int32_t n_rsb, n_tiles;                  // tiles = n_rsb x ceil(M / BN); tile t -> (t % n_rsb, t / n_rsb)
 };
 
 struct GemmPlan {
     int32_t dummy;
 };
 
+#ifdef QL_TRACE
+// Developer aid (not compiled by default): %globaltimer stamps of the first k-steps of CTAs 0 and 1.
+constexpr int kGTraceSteps = 48, kGTraceEvents = 8;
+__device__ unsigned long long g_gemm_trace[2][kGTraceEvents][kGTraceSteps];
+__device__ __forceinline__ void gemm_trace(int ev, int step)
+{
+    if (blockIdx.x < 2 && step < kGTraceSteps) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        g_gemm_trace[blockIdx.x][ev][step] = t;
+    }
+}
+#define QL_GTRACE(ev, step) gemm_trace(ev, step)
+#else
+#define QL_GTRACE(ev, step) do { } while (0)
+#endif
+
+// Per-lane constants and the per-step work of a dequantise warp (shared by the 1-CTA and 2-CTA kernels).
+// Warp dw handles row-block (dw & 7); of each lane's 16 packed bytes (two 32-wide k halves) a lane
+// converts one half per step: half (dw >> 3) for even g, the other one for odd g; the partner warp
+// (dw ^ 8) takes the rest.  Swizzled, the 8 lanes of a quarter-warp then store to 8 different 16-byte
+// columns: no bank conflicts.
+struct DequantLane {
+    int half;
+    uint32_t off_lo, off_hi, s_sel;
+    int w_off4, w_off8, s_off;
+    __device__ DequantLane(int dw, int lane)
+    {
+        const int g = lane >> 2, c = lane & 3;
+        const int row0 = (dw & 7) * kRbRows + g;                         // rows row0 and row0 + 8 ((row & 7) == g)
+        half = (dw >> 3) ^ (g & 1);                                      // which 32-k half of the 64-k step
+        const uint32_t unit = ((uint32_t)(4 * half + c) ^ (uint32_t)g) * 16;
+        off_lo = row0 * 128 + unit;
+        off_hi = (row0 + 8) * 128 + unit;
+        w_off4 = (dw & 7) * 512 + lane * 16 + 8 * half;
+        w_off8 = half * kWeightBlockBytes + (dw & 7) * 512 + lane * 16;
+        s_off = kWeightBlockBytes + (dw & 7) * 64 + g * 8;
+        s_sel = half ? 0x3232u : 0x1010u;                                // broadcast the scale of this half's group
+    }
+    template <int BITS, bool GROUPED>
+    __device__ __forceinline__ void step(const unsigned char* wp, unsigned char* at) const
+    {
+        uint32_t a0[4], a1[4];
+        if (BITS == 4) {
+            const uint2 w = *reinterpret_cast<const uint2*>(wp + w_off4);
+            unpack_int4_word(w.x, a0);                                   // k 32*half + 8c     .. + 3
+            unpack_int4_word(w.y, a1);                                   // k 32*half + 8c + 4 .. + 7
+        } else {
+            const uint4 w = *reinterpret_cast<const uint4*>(wp + w_off8);
+            unpack_int8_words(w.x, w.y, a0);
+            unpack_int8_words(w.z, w.w, a1);
+        }
+        uint4 lo = make_uint4(a0[0], a0[2], a1[0], a1[2]);               // row0
+        uint4 hi = make_uint4(a0[1], a0[3], a1[1], a1[3]);               // row0 + 8
+        if (GROUPED) {
+            const uint2 sc = *reinterpret_cast<const uint2*>(wp + s_off);
+            const uint32_t s_lo = __byte_perm(sc.x, 0, s_sel), s_hi = __byte_perm(sc.y, 0, s_sel);
+            lo.x = h2_mul(lo.x, s_lo); lo.y = h2_mul(lo.y, s_lo); lo.z = h2_mul(lo.z, s_lo); lo.w = h2_mul(lo.w, s_lo);
+            hi.x = h2_mul(hi.x, s_hi); hi.y = h2_mul(hi.y, s_hi); hi.z = h2_mul(hi.z, s_hi); hi.w = h2_mul(hi.w, s_hi);
+        }
+        *reinterpret_cast<uint4*>(at + off_lo) = lo;
+        *reinterpret_cast<uint4*>(at + off_hi) = hi;
+    }
+};
+
 // ----------------------------------------------------------------------------- shared-memory plan
 template <int BITS, int BN>
 struct GemmSmem {
-    static constexpr int kWpkBytes = BITS == 4 ? (kWeightBlockBytes + kScaleBlockBytes) : 2 * kWeightBlockBytes;
     static constexpr int kWpkStride = 8192;                              // keeps every tile 1024-byte aligned
     static constexpr int kXBytes = BN * 128;
     static constexpr int kStageBytes = kXBytes + kGemmATileBytes + kWpkStride;
@@ -74,16 +142,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     auto wpk_ptr = [&](int s) { return base_ptr + s * S::kStageBytes + S::kXBytes + kGemmATileBytes; };
     auto a_ptr = [&](int s) { return base_ptr + s * S::kStageBytes + S::kXBytes; };
     const uint32_t bar0 = base + S::kBarOffset;
-    auto full_bar = [&](int s) { return bar0 + 8 * s; };
-    auto afull_bar = [&](int s) { return bar0 + 8 * (NS + s); };
-    auto empty_bar = [&](int s) { return bar0 + 8 * (2 * NS + s); };
-    const uint32_t accum_bar = bar0 + 8 * (3 * NS);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kBarOffset + 8 * (3 * NS + 1));
+    auto full_bar = [&](int s) { return bar0 + 8 * s; };                 // TMA data of stage s landed
+    auto afull_bar = [&](int s) { return bar0 + 8 * (NS + s); };         // A tile of stage s dequantised
+    auto empty_bar = [&](int s) { return bar0 + 8 * (2 * NS + s); };     // MMAs of stage s retired
+    auto tfull_bar = [&](int b) { return bar0 + 8 * (3 * NS + b); };     // accumulator b complete
+    auto tempty_bar = [&](int b) { return bar0 + 8 * (3 * NS + 2 + b); };// accumulator b drained by the epilogue
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kBarOffset + 8 * (3 * NS + 4));
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int rsb = blockIdx.x, m0 = blockIdx.y * BN;
     const int n_steps = p.n_ksteps;
+    const int first_tile = blockIdx.x, tile_stride = gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
@@ -91,12 +160,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(afull_bar(s), kGemmDequantWarps);
             mbar_init(empty_bar(s), 1);
         }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), kGemmEpilogueWarps);
+        }
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), BN);
+    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), 2 * BN);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -107,23 +179,28 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
             constexpr int CHUNKS = BITS == 4 ? 1 : 2;                    // packed blocks per 64-k step
-            const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
-            int issued = 0;
-            bool waited_dep = false;
-            for (int it = 0; it < n_steps; ++it) {
-                const int s = it % NS, r = it / NS;
-                if (!mbar_wait(empty_bar(s), (r & 1) ^ 1, abort_flag, 0x100 + s)) break;
-                const int kc = it * CHUNKS;
-                const int nblk = min(CHUNKS, p.n_kc - kc);
-                const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
-                mbar_expect_tx(full_bar(s), wbytes + S::kXBytes);
-                bulk_copy_g2s(wpk_addr(s), wsrc + (int64_t)kc * p.block_bytes, wbytes, full_bar(s));
-                if (!waited_dep) {                                       // x may come from the previous kernel
-                    asm volatile("griddepcontrol.wait;" ::: "memory");
-                    waited_dep = true;
+            int s = 0, issued = 0;
+            uint32_t par = 1;                                            // first pass: stages start out free
+            bool waited_dep = false, ok = true;
+            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+                const int rsb = t % p.n_rsb, m0 = (t / p.n_rsb) * BN;
+                const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
+                for (int it = 0; it < n_steps; ++it) {
+                    if (!mbar_wait(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
+                    QL_GTRACE(0, issued);
+                    const int kc = it * CHUNKS;
+                    const int nblk = min(CHUNKS, p.n_kc - kc);
+                    const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
+                    mbar_expect_tx(full_bar(s), wbytes + S::kXBytes);
+                    bulk_copy_g2s(wpk_addr(s), wsrc + (int64_t)kc * p.block_bytes, wbytes, full_bar(s));
+                    if (!waited_dep) {                                   // x may come from the previous kernel
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        waited_dep = true;
+                    }
+                    tma_load_2d(xs_addr(s), &x_map, it * kGemmKStep, m0, full_bar(s));
+                    ++issued;
+                    if (++s == NS) { s = 0; par ^= 1; }
                 }
-                tma_load_2d(xs_addr(s), &x_map, it * kGemmKStep, m0, full_bar(s));
-                ++issued;
             }
             if (*abort_flag) {                                           // let copies in flight land before exit
                 for (int j = max(0, issued - NS); j < issued; ++j)
@@ -134,105 +211,91 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_f16(BN);
+            const uint32_t a_lo0 = umma_desc_lo(a_addr(0)), b_lo0 = umma_desc_lo(xs_addr(0));
+            int s = 0;
+            uint32_t par = 0;
             bool ok = true;
-            for (int it = 0; it < n_steps && ok; ++it) {
-                const int s = it % NS, r = it / NS;
-                ok = mbar_wait(full_bar(s), r & 1, abort_flag, 0x200 + s) &&
-                     mbar_wait(afull_bar(s), r & 1, abort_flag, 0x300 + s);
-                if (!ok) break;
+            int j = 0;                                                   // local tile counter
+            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+                const int buf = j & 1;
+                const uint32_t use = (uint32_t)(j >> 1);
+                // accumulator buf must have been drained by the epilogue of its previous use
+                if (!mbar_wait(tempty_bar(buf), (use & 1) ^ 1, abort_flag, 0x800 + buf)) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                for (int it = 0; it < n_steps; ++it) {
+                    // A tile written; the dequantise warps waited for the stage's TMA data, so x landed too
+                    ok = mbar_wait(afull_bar(s), par, abort_flag, 0x300 + s);
+                    if (!ok) break;
+                    QL_GTRACE(5, j * n_steps + it);
+                    tc_fence_after();
+                    const uint32_t a_lo = a_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
+                    umma_f16_lo(tmem_d, a_lo, b_lo, idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-                for (int k4 = 0; k4 < kGemmKStep / 16; ++k4) {
-                    const uint64_t ad = umma_desc_sw128(a_addr(s) + k4 * 32);
-                    const uint64_t bd = umma_desc_sw128(xs_addr(s) + k4 * 32);
-                    umma_f16(tmem_base, ad, bd, idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                    for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)         // +32 bytes along K inside the swizzle row
+                        umma_f16_lo(tmem_d, a_lo + 2 * k4, b_lo + 2 * k4, idesc, 1u);
+                    umma_commit(empty_bar(s));
+                    QL_GTRACE(6, j * n_steps + it);
+                    if (++s == NS) { s = 0; par ^= 1; }
                 }
-                umma_commit(empty_bar(s));
+                umma_commit(tfull_bar(buf));
             }
-            umma_commit(accum_bar);
+        }
+    } else if (warp < 2 + kGemmDequantWarps) {
+        // ------------------------------------------------------------------ dequantise
+        // Warp dw handles row-block (dw & 7); of each lane's 16 packed bytes (two 32-wide k halves) a
+        // lane converts one half per step: half (dw >> 3) for even g, the other one for odd g, the
+        // partner warp (dw ^ 8) takes the rest.  Swizzled, the 8 lanes of a quarter-warp then store to
+        // 8 different 16-byte columns: no bank conflicts.
+        const DequantLane dq(warp - 2, lane);
+        int s = 0;
+        uint32_t par = 0;
+        bool ok = true;
+        int gstep = 0;
+        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+            for (int it = 0; it < n_steps; ++it, ++gstep) {
+                if (!mbar_wait(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
+                if (threadIdx.x == 64) QL_GTRACE(1, gstep);
+                dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(s));
+                fence_async_smem();                                      // generic-proxy writes -> visible to the MMA
+                __syncwarp();
+                if (threadIdx.x == 64) QL_GTRACE(3, gstep);
+                if (lane == 0) mbar_arrive(afull_bar(s));
+                if (++s == NS) { s = 0; par ^= 1; }
+            }
         }
     } else {
-        // ------------------------------------------------------------------ dequantise, then epilogue
-        const int dw = warp - 2;                                         // 0..7 = row-block of the tile
-        const int g = lane >> 2, c = lane & 3;
-        const int row0 = dw * kRbRows + g;                               // rows row0 and row0 + 8
-        const uint32_t sw = (uint32_t)g;                                 // (row & 7) of both rows
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                                    // TMEM lanes 32*quarter .. +31
         bool ok = true;
-        for (int it = 0; it < n_steps && ok; ++it) {
-            const int s = it % NS, r = it / NS;
-            ok = mbar_wait(full_bar(s), r & 1, abort_flag, 0x400 + s);
-            if (!ok) break;
-            const unsigned char* wp = wpk_ptr(s);
-            unsigned char* at = a_ptr(s);
-            if (BITS == 4) {
-                const uint4 w = *reinterpret_cast<const uint4*>(wp + dw * 512 + lane * 16);
-                uint32_t lo[4], hi[4];                                   // words 0,1 -> k 8c..8c+7; words 2,3 -> 32+8c..
-                uint32_t a0[4], a1[4];
-                unpack_int4_word(w.x, a0);
-                unpack_int4_word(w.y, a1);
-                lo[0] = a0[0]; lo[1] = a0[2]; lo[2] = a1[0]; lo[3] = a1[2];        // row0,   unit c
-                hi[0] = a0[1]; hi[1] = a0[3]; hi[2] = a1[1]; hi[3] = a1[3];        // row0+8, unit c
-                uint32_t lo2[4], hi2[4];
-                unpack_int4_word(w.z, a0);
-                unpack_int4_word(w.w, a1);
-                lo2[0] = a0[0]; lo2[1] = a0[2]; lo2[2] = a1[0]; lo2[3] = a1[2];    // row0,   unit 4+c
-                hi2[0] = a0[1]; hi2[1] = a0[3]; hi2[2] = a1[1]; hi2[3] = a1[3];    // row0+8, unit 4+c
-                if (GROUPED) {
-                    const uint2 sc = *reinterpret_cast<const uint2*>(wp + kWeightBlockBytes + dw * 64 + g * 8);
-                    const uint32_t s_g0 = __byte_perm(sc.x, 0, 0x1010), s_g1 = __byte_perm(sc.x, 0, 0x3232);
-                    const uint32_t s_h0 = __byte_perm(sc.y, 0, 0x1010), s_h1 = __byte_perm(sc.y, 0, 0x3232);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        lo[i] = h2_mul(lo[i], s_g0);  lo2[i] = h2_mul(lo2[i], s_g1);
-                        hi[i] = h2_mul(hi[i], s_h0);  hi2[i] = h2_mul(hi2[i], s_h1);
-                    }
-                }
-                const uint32_t u0 = ((uint32_t)c ^ sw) * 16, u1 = ((uint32_t)(4 + c) ^ sw) * 16;
-                *reinterpret_cast<uint4*>(at + row0 * 128 + u0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                *reinterpret_cast<uint4*>(at + row0 * 128 + u1) = make_uint4(lo2[0], lo2[1], lo2[2], lo2[3]);
-                *reinterpret_cast<uint4*>(at + (row0 + 8) * 128 + u0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                *reinterpret_cast<uint4*>(at + (row0 + 8) * 128 + u1) = make_uint4(hi2[0], hi2[1], hi2[2], hi2[3]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {                            // two 32-k chunks per step
-                    const uint4 w = *reinterpret_cast<const uint4*>(wp + j * kWeightBlockBytes + dw * 512 + lane * 16);
-                    uint32_t a0[4], a1[4];
-                    unpack_int8_words(w.x, w.y, a0);
-                    unpack_int8_words(w.z, w.w, a1);
-                    const uint32_t u = ((uint32_t)(4 * j + c) ^ sw) * 16;
-                    *reinterpret_cast<uint4*>(at + row0 * 128 + u) = make_uint4(a0[0], a0[2], a1[0], a1[2]);
-                    *reinterpret_cast<uint4*>(at + (row0 + 8) * 128 + u) = make_uint4(a0[1], a0[3], a1[1], a1[3]);
-                }
-            }
-            fence_async_smem();                                          // generic-proxy writes -> visible to the MMA
-            __syncwarp();
-            if (lane == 0) mbar_arrive(afull_bar(s));
-        }
-
-        // epilogue: warp (dw & 3) + 2 owns the TMEM lane quarter (warp % 4); two warps split the columns
-        if (ok) ok = mbar_wait(accum_bar, 0, abort_flag, 0x500);
-        if (ok) {
+        int j = 0;
+        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+            const int buf = j & 1;
+            const uint32_t use = (uint32_t)(j >> 1);
+            const int rsb = t % p.n_rsb, m0 = (t / p.n_rsb) * BN;
+            if (!mbar_wait(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
-            const int quarter = warp & 3;
-            const int half = dw >> 2;
             const int n = rsb * kRsbRows + quarter * 32 + lane;
             float scale = 1.f;
             if (!GROUPED && n < p.N) scale = __half2float(p.chan_scales[n]);
-            constexpr int CW = BN / 2;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+            __half* yrow = p.y + (int64_t)m0 * p.N + n;
+            const int m_left = p.M - m0;
 #pragma unroll 1
-            for (int cc = 0; cc < CW; cc += 16) {
-                const int col0 = half * CW + cc;
-                if (m0 + col0 >= p.M) break;
+            for (int cc = 0; cc < BN; cc += 16) {
+                if (cc >= m_left) break;
                 uint32_t r[16];
-                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col0, r);
+                tmem_ld16(taddr + (uint32_t)cc, r);
                 if (n < p.N) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int m = m0 + col0 + j;
-                        if (m < p.M) p.y[(int64_t)m * p.N + n] = __float2half_rn(__uint_as_float(r[j]) * scale);
-                    }
+                    for (int q = 0; q < 16; ++q)
+                        if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(__uint_as_float(r[q]) * scale);
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
         }
     }
 
@@ -240,7 +303,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, BN);
+        tmem_dealloc(tmem_base, 2 * BN);
     }
 }
 
@@ -286,7 +349,7 @@ inline int gemm_pick_bn(const Layout& L, int M, int num_sms)
 }
 
 template <int BITS, bool GROUPED, int BN>
-ql_status gemm_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device, bool pdl)
+ql_status gemm_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device, bool pdl, int num_sms)
 {
     using S = GemmSmem<BITS, BN>;
     static_assert(S::kStages >= 2, "pipeline needs at least two stages");
@@ -318,9 +381,11 @@ ql_status gemm_launch(const Layout& L, const uint8_t* blob, const void* x, void*
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
+    prm.n_rsb = L.n_rsb;
+    prm.n_tiles = L.n_rsb * ((M + BN - 1) / BN);
 
     cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(L.n_rsb, (M + BN - 1) / BN);
+    cfg.gridDim = dim3(prm.n_tiles < num_sms ? prm.n_tiles : num_sms);
     cfg.blockDim = dim3(kGemmThreads);
     cfg.dynamicSmemBytes = S::kTotal;
     cfg.stream = st;
@@ -338,13 +403,13 @@ ql_status gemm_launch(const Layout& L, const uint8_t* blob, const void* x, void*
 
 template <int BITS, bool GROUPED>
 ql_status gemm_dispatch_bn(int bn, const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st,
-                           int device, bool pdl)
+                           int device, bool pdl, int num_sms)
 {
     switch (bn) {
-        case 32: return gemm_launch<BITS, GROUPED, 32>(L, blob, x, y, M, st, device, pdl);
-        case 64: return gemm_launch<BITS, GROUPED, 64>(L, blob, x, y, M, st, device, pdl);
-        case 128: return gemm_launch<BITS, GROUPED, 128>(L, blob, x, y, M, st, device, pdl);
-        case 256: return gemm_launch<BITS, GROUPED, 256>(L, blob, x, y, M, st, device, pdl);
+        case 32: return gemm_launch<BITS, GROUPED, 32>(L, blob, x, y, M, st, device, pdl, num_sms);
+        case 64: return gemm_launch<BITS, GROUPED, 64>(L, blob, x, y, M, st, device, pdl, num_sms);
+        case 128: return gemm_launch<BITS, GROUPED, 128>(L, blob, x, y, M, st, device, pdl, num_sms);
+        case 256: return gemm_launch<BITS, GROUPED, 256>(L, blob, x, y, M, st, device, pdl, num_sms);
     }
     return QL_ERR_INVALID_ARG;
 }
@@ -353,9 +418,9 @@ inline ql_status gemm_forward(const Layout& L, const GemmPlan&, const uint8_t* b
                               cudaStream_t st, int device, bool pdl, int num_sms)
 {
     const int bn = gemm_pick_bn(L, M, num_sms);
-    if (L.bits == 8) return gemm_dispatch_bn<8, false>(bn, L, blob, x, y, M, st, device, pdl);
-    if (L.grouped) return gemm_dispatch_bn<4, true>(bn, L, blob, x, y, M, st, device, pdl);
-    return gemm_dispatch_bn<4, false>(bn, L, blob, x, y, M, st, device, pdl);
+    if (L.bits == 8) return gemm_dispatch_bn<8, false>(bn, L, blob, x, y, M, st, device, pdl, num_sms);
+    if (L.grouped) return gemm_dispatch_bn<4, true>(bn, L, blob, x, y, M, st, device, pdl, num_sms);
+    return gemm_dispatch_bn<4, false>(bn, L, blob, x, y, M, st, device, pdl, num_sms);
 }
 
 }  // namespace ql

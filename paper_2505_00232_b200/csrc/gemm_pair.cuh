@@ -1,0 +1,326 @@
+// Prefill kernel, CTA-pair form (tcgen05 cta_group::2): two CTAs of a cluster compute one 256 x 256 output
+// tile -- 256 output channels (two row super-blocks, one per CTA) x 256 tokens -- with one MMA issued by
+// the leader CTA.  Each CTA stages only its own 128 channels of weights and its own 128 tokens of x, so
+// the x traffic from L2 and the shared-memory operand reads per flop are half of the single-CTA kernel's
+// (paper Section 3.7: the prefill stage is compute-bound; the point here is to keep it that way).
+//
+// Roles per CTA are those of gemm.cuh.  Cross-CTA protocol (no TMA multicast anywhere):
+//   * dequantise warps arrive on their own CTA's afull barrier (a warp dequantises only after its CTA's
+//     TMA data landed, so "A tile written" implies "x half landed"); in the peer CTA the otherwise idle
+//     MMA warp relays each completed afull phase to the leader with ONE remote arrive, on the leader's
+//     afull barrier (17 arrivals there: its own 16 warps and the relay);
+//   * the leader's tcgen05.commit signals the empty / tfull barriers of BOTH CTAs (commit multicast);
+//   * the epilogue warps of both CTAs arrive on the leader's tempty barrier (8 arrivals);
+//   * cluster barriers bracket the kernel so that no CTA exits while its peer can still touch it.
+#pragma once
+#include "gemm.cuh"
+
+namespace ql {
+
+// Shared memory: a deep ring of TMA stages (this CTA's x half + packed weights) that covers the load
+// latency, and a short ring of dequantised A tiles (produced on chip, consumed a few hundred cycles later).
+// Warp roles: 0 producer, 1 MMA / relay, 2..22 except ids with (id % 4 == 1): 16 dequantise warps, 24..27 epilogue.
+constexpr int kPairFirstEpilogueWarp = 24;
+constexpr int kPairThreads = 28 * 32;
+
+template <int BITS>
+struct GemmPairSmem {
+    static constexpr int kXBytes = 128 * 128;                            // this CTA's 128 tokens x 64 k
+    static constexpr int kWpkStride = BITS == 4 ? 5120 : 8192;           // packed block(s) of one k-step
+    static constexpr int kStageBytes = kXBytes + kWpkStride;
+    static constexpr int kStages = 6;
+    static constexpr int kASlots = 4;
+    static constexpr int kAOffset = kStages * kStageBytes;
+    static constexpr int kBarOffset = kAOffset + kASlots * kGemmATileBytes;
+    static constexpr int kTotal = kBarOffset + 512 + 1024;               // barriers + alignment slack
+};
+
+template <int BITS, bool GROUPED>
+__global__ void __launch_bounds__(kPairThreads, 1)
+gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
+{
+    using S = GemmPairSmem<BITS>;
+    constexpr int NS = S::kStages;
+    constexpr int NA = S::kASlots;
+    constexpr int BN = 256;                                              // tokens per tile (128 per CTA)
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    auto xs_addr = [&](int s) { return base + s * S::kStageBytes; };
+    auto wpk_addr = [&](int s) { return base + s * S::kStageBytes + S::kXBytes; };
+    auto wpk_ptr = [&](int s) { return base_ptr + s * S::kStageBytes + S::kXBytes; };
+    auto a_addr = [&](int a) { return base + S::kAOffset + a * kGemmATileBytes; };
+    auto a_ptr = [&](int a) { return base_ptr + S::kAOffset + a * kGemmATileBytes; };
+    const uint32_t bar0 = base + S::kBarOffset;
+    auto full_bar = [&](int s) { return bar0 + 8 * s; };                 // local: this CTA's TMA data landed
+    auto empty_bar = [&](int s) { return bar0 + 8 * (NS + s); };         // local, signalled by the leader's commit
+    auto afull_bar = [&](int a) { return bar0 + 8 * (2 * NS + a); };     // local: this CTA's A tile written
+    auto aempty_bar = [&](int a) { return bar0 + 8 * (2 * NS + NA + a); };   // local, signalled by the leader's commit
+    auto pready_bar = [&](int a) { return bar0 + 8 * (2 * NS + 2 * NA + a); };   // leader: the peer's A slot is ready
+    auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + 3 * NA + b); };        // local, signalled by the leader's commit
+    auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 3 * NA + 2 + b); };   // leader: both epilogues drained buffer b
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kBarOffset + 8 * (2 * NS + 3 * NA + 4));
+    volatile uint32_t* abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                             // 0 = leader
+    const int n_steps = p.n_ksteps;
+    const int n_pairs = p.n_rsb >> 1;
+    const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < NA; ++a) {
+            mbar_init(afull_bar(a), kGemmDequantWarps + (rank == 0 ? 1 : 0));   // leader: + the peer's relay lane
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull_bar(b), 1);
+            mbar_init(tempty_bar(b), 2 * kGemmEpilogueWarps);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32((const void*)tmem_slot), 2 * BN);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                                  // both CTAs' barriers exist before any remote arrive
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer (each CTA feeds itself)
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
+            constexpr int CHUNKS = BITS == 4 ? 1 : 2;
+            int s = 0, issued = 0;
+            uint32_t par = 1;
+            bool waited_dep = false, ok = true;
+            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+                const int rsb = 2 * (t % n_pairs) + (int)rank;
+                const int m0 = (t / n_pairs) * BN + 128 * (int)rank;     // this CTA's 128 tokens of the tile
+                const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
+                for (int it = 0; it < n_steps; ++it) {
+                    if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
+                    QL_GTRACE(0, issued);
+                    const int kc = it * CHUNKS;
+                    const int nblk = min(CHUNKS, p.n_kc - kc);
+                    const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
+                    mbar_expect_tx(full_bar(s), wbytes + S::kXBytes);
+                    bulk_copy_g2s(wpk_addr(s), wsrc + (int64_t)kc * p.block_bytes, wbytes, full_bar(s));
+                    if (!waited_dep) {
+                        asm volatile("griddepcontrol.wait;" ::: "memory");
+                        waited_dep = true;
+                    }
+                    tma_load_2d(xs_addr(s), &x_map, it * kGemmKStep, m0, full_bar(s));
+                    ++issued;
+                    if (++s == NS) { s = 0; par ^= 1; }
+                }
+            }
+            if (*abort_flag) {
+                for (int j = max(0, issued - NS); j < issued; ++j)
+                    mbar_wait(full_bar(j % NS), (j / NS) & 1, abort_flag + 1, 0);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            const uint32_t a_lo0 = umma_desc_lo(a_addr(0)), b_lo0 = umma_desc_lo(xs_addr(0));
+            int s = 0, a = 0;
+            uint32_t apar = 0;
+            bool ok = true;
+            int j = 0;
+            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+                const int buf = j & 1;
+                const uint32_t use = (uint32_t)(j >> 1);
+                if (!mbar_wait(tempty_bar(buf), (use & 1) ^ 1, abort_flag, 0x800 + buf)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
+                for (int it = 0; it < n_steps; ++it) {
+                    // own A tile written (implies own x half landed) and the peer's likewise
+                    // 16 local dequantise warps + the peer's relay lane: both A tiles written, both x halves landed
+                    if (!mbar_wait(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
+                    QL_GTRACE(5, j * n_steps + it);
+                    tc_fence_after();
+                    const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
+                    const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
+                    umma_f16_pair_lo(tmem_d, a_lo, b_lo, idesc, it > 0 ? 1u : 0u);
+#pragma unroll
+                    for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)
+                        umma_f16_pair_lo(tmem_d, a_lo + 2 * k4, b_lo + 2 * k4, idesc, 1u);
+                    umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
+                    QL_GTRACE(6, j * n_steps + it);
+                    if (++s == NS) s = 0;
+                    if (++a == NA) { a = 0; apar ^= 1; }
+                }
+                if (ok) umma_commit_pair(tfull_bar(buf));
+            }
+        }
+    } else if (warp < kPairFirstEpilogueWarp) {
+        // ------------------------------------------------------------------ dequantise
+        // The MMA-issuing warp (warp 1) lives on scheduler 1 (warp id % 4); dequantise work is kept off
+        // that scheduler so that the issuing thread is never queued behind ALU-heavy warps.
+        if ((warp & 3) == 1) {
+            // Spare warps 5, 9, 13, 17 of the PEER CTA relay "A slot ready" to the leader: one warp per A
+            // slot (a waiting warp is suspended as a whole, so relay lanes of one warp would serialise),
+            // one remote arrive per slot phase on the leader's afull barrier.
+            const int a = (warp - 5) >> 2;
+            if (rank != 0 && lane == 0 && a < NA) {
+                uint32_t apar = 0;
+                const int total_steps = n_steps * ((p.n_tiles - first_tile + tile_stride - 1) / tile_stride);
+                for (int g = a; g < total_steps; g += NA) {
+                    if (!mbar_wait(afull_bar(a), apar, abort_flag, 0xA00 + a)) break;
+                    mbar_arrive_remote(afull_bar(a), 0);
+                    apar ^= 1;
+                }
+            }
+        } else if (warp <= 22) {                                         // 16 dequantise warps; warp 23 idles
+        const DequantLane dq(warp - 2 - ((warp - 1) >> 2), lane);
+        int s = 0, a = 0;
+        uint32_t par = 0;
+        // A slot a was last read by the MMAs of step (gstep - NA); their retirement is the phase of the
+        // empty barrier of that step's TMA stage.
+        int s_old = 0;
+        uint32_t par_old = 0;
+        bool ok = true;
+        int gstep = 0;
+        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+            for (int it = 0; it < n_steps; ++it, ++gstep) {
+                if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
+                if (threadIdx.x == 64) QL_GTRACE(1, gstep);
+                if (gstep >= NA) {
+                    if (!mbar_wait(empty_bar(s_old), par_old, abort_flag, 0xB00 + s_old)) { ok = false; break; }
+                    if (++s_old == NS) { s_old = 0; par_old ^= 1; }
+                }
+                if (threadIdx.x == 64) QL_GTRACE(2, gstep);
+                dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(a));
+                fence_async_smem();
+                __syncwarp();
+                if (threadIdx.x == 64) QL_GTRACE(3, gstep);
+                if (lane == 0) mbar_arrive(afull_bar(a));
+                if (++s == NS) { s = 0; par ^= 1; }
+                if (++a == NA) a = 0;
+            }
+        }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (each CTA stores its 128 channels)
+        const int quarter = warp & 3;
+        bool ok = true;
+        int j = 0;
+        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+            const int buf = j & 1;
+            const uint32_t use = (uint32_t)(j >> 1);
+            const int rsb = 2 * (t % n_pairs) + (int)rank, m0 = (t / n_pairs) * BN;
+            if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
+            tc_fence_after();
+            const int n = rsb * kRsbRows + quarter * 32 + lane;
+            float scale = 1.f;
+            if (!GROUPED && n < p.N) scale = __half2float(p.chan_scales[n]);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+            __half* yrow = p.y + (int64_t)m0 * p.N + n;
+            const int m_left = p.M - m0;
+#pragma unroll 1
+            for (int cc = 0; cc < BN; cc += 16) {
+                if (cc >= m_left) break;
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)cc, r);
+                if (n < p.N) {
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(__uint_as_float(r[q]) * scale);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                                  // the peer no longer reads this CTA's memory
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, 2 * BN);
+    }
+}
+
+template <int BITS, bool GROUPED>
+ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device,
+                           bool pdl, int num_sms)
+{
+    using S = GemmPairSmem<BITS>;
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return QL_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t gdim[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
+    const cuuint64_t gstr[1] = {(cuuint64_t)L.K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kGemmKStep, 128u};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return QL_ERR_CUDA;
+    auto kern = gemm_pair_kernel<BITS, GROUPED>;
+    static bool attr_set[64] = {};
+    if (device >= 0 && device < 64 && !attr_set[device]) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
+            cudaGetLastError();
+            return QL_ERR_CUDA;
+        }
+        attr_set[device] = true;
+    }
+    GemmParams prm{};
+    prm.body = blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(blob + L.chan_scale_offset);
+    prm.y = static_cast<__half*>(y);
+    prm.M = M; prm.N = L.N; prm.K = L.K;
+    prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
+    prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
+    prm.n_rsb = L.n_rsb;
+    prm.n_tiles = (L.n_rsb / 2) * ((M + 255) / 256);
+    const int n_clusters = prm.n_tiles < num_sms / 2 ? prm.n_tiles : num_sms / 2;
+
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2 * n_clusters);
+    cfg.blockDim = dim3(kPairThreads);
+    cfg.dynamicSmemBytes = S::kTotal;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kern, map, prm) != cudaSuccess) {
+        cudaGetLastError();
+        return QL_ERR_CUDA;
+    }
+    return QL_OK;
+}
+
+// The pair kernel needs an even number of row super-blocks and enough tokens to fill a 256-wide tile.
+inline bool gemm_pair_applicable(const Layout& L, int M)
+{
+    const char* f = std::getenv("QLINEAR_GEMM_PAIR");
+    if (f && *f == '0') return false;
+    return (L.n_rsb % 2) == 0 && M > 128;
+}
+
+inline ql_status gemm_pair_forward(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st,
+                                   int device, bool pdl, int num_sms)
+{
+    if (L.bits == 8) return gemm_pair_launch<8, false>(L, blob, x, y, M, st, device, pdl, num_sms);
+    if (L.grouped) return gemm_pair_launch<4, true>(L, blob, x, y, M, st, device, pdl, num_sms);
+    return gemm_pair_launch<4, false>(L, blob, x, y, M, st, device, pdl, num_sms);
+}
+
+}  // namespace ql

@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
             int s = 0;                                                   // pro == NS whenever this loop runs
             uint32_t par = 0;                                            // parity of the consumers' first release
             for (int i = pro; i < nb; ++i) {
-                if (!mbar_wait(empty_bar(s), par, abort_flag, 0x600 + s)) break;
+                if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x600 + s)) break;
                 issue_w(i, s);
                 issue_x(s, kcp);
                 kcp = kcp + 1 == p.n_kc ? 0 : kcp + 1;
@@ -289,8 +289,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
 #pragma unroll
         for (int s = 0; s < NS; s += 2) {
             if (j >= npairs) break;
-            if (!mbar_wait(full_bar(s), par, abort_flag, 0x700 + s)) return;
-            if (!mbar_wait(full_bar(s + 1), par, abort_flag, 0x700 + s + 1)) return;
+            if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x700 + s)) return;
+            if (!mbar_wait<true>(full_bar(s + 1), par, abort_flag, 0x700 + s + 1)) return;
             if (j == 0 && threadIdx.x == 0) QL_TRACE_AT(p.trace_seq, 3);
             StreamFrag fa, fb;
             stream_load<BITS, GROUPED>(fa, smem_dyn + s * ST::kBytes, w_off, s_off, x_off);
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
     if (nb & 1) {                                                        // odd range: one more block
         const int s = (nb - 1) % NS;
         const uint32_t par_last = (uint32_t)((nb - 1) / NS) & 1u;
-        if (!mbar_wait(full_bar(s), par_last, abort_flag, 0x700 + s)) return;
+        if (!mbar_wait<true>(full_bar(s), par_last, abort_flag, 0x700 + s)) return;
         StreamFrag fa;
         stream_load<BITS, GROUPED>(fa, smem_dyn + s * ST::kBytes, w_off, s_off, x_off);
         stream_math<BITS, GROUPED>(fa, total);

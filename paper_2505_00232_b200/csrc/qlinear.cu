@@ -21,6 +21,7 @@ __device__ unsigned int g_device_flag[2];
 #include "gemv.cuh"
 #include "gemv_stream.cuh"
 #include "gemm.cuh"
+#include "gemm_pair.cuh"
 
 using namespace ql;
 
@@ -306,6 +307,7 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(h, x, y, M, st);
+    if (gemm_pair_applicable(h->L, M)) return gemm_pair_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
     return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
@@ -366,6 +368,10 @@ extern "C" const char* qlinear_status_string(ql_status s)
 }
 
 #ifdef QL_TRACE
+extern "C" int qlinear_debug_read_gemm_trace(unsigned long long* out, size_t bytes)
+{
+    return (int)cudaMemcpyFromSymbol(out, g_gemm_trace, bytes < sizeof(g_gemm_trace) ? bytes : sizeof(g_gemm_trace));
+}
 extern "C" int qlinear_debug_read_trace(unsigned long long* out, size_t bytes)
 {
     return (int)cudaMemcpyFromSymbol(out, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
