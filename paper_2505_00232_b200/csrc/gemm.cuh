@@ -55,9 +55,13 @@ struct GemmPlan {
 // Developer aid (not compiled by default): %globaltimer stamps of the first k-steps of CTAs 0 and 1.
 constexpr int kGTraceSteps = 48, kGTraceEvents = 8;
 __device__ unsigned long long g_gemm_trace[2][kGTraceEvents][kGTraceSteps];
+#ifndef QL_TRACE_OFFSET
+#define QL_TRACE_OFFSET 0
+#endif
 __device__ __forceinline__ void gemm_trace(int ev, int step)
 {
-    if (blockIdx.x < 2 && step < kGTraceSteps) {
+    step -= QL_TRACE_OFFSET;                                             // first recorded k-step of the CTA
+    if (blockIdx.x < 2 && step >= 0 && step < kGTraceSteps) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         g_gemm_trace[blockIdx.x][ev][step] = t;

@@ -28,8 +28,8 @@ struct GemmPairSmem {
     static constexpr int kXBytes = 128 * 128;                            // this CTA's 128 tokens x 64 k
     static constexpr int kWpkStride = BITS == 4 ? 5120 : 8192;           // packed block(s) of one k-step
     static constexpr int kStageBytes = kXBytes + kWpkStride;
-    static constexpr int kStages = 6;
-    static constexpr int kASlots = 4;
+    static constexpr int kStages = BITS == 4 ? 6 : 5;
+    static constexpr int kASlots = 5;                                    // one relay warp per slot (warps 5, 9, 13, 17, 21, 23)
     static constexpr int kAOffset = kStages * kStageBytes;
     static constexpr int kBarOffset = kAOffset + kASlots * kGemmATileBytes;
     static constexpr int kTotal = kBarOffset + 512 + 1024;               // barriers + alignment slack
@@ -65,7 +65,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                             // 0 = leader
     const int n_steps = p.n_ksteps;
-    const int n_pairs = p.n_rsb >> 1;
+    // Tile t = (row-super-block pair t / n_mblk, token block t % n_mblk): clusters that run side by side share
+    // weight blocks and read different x tiles, which spreads the L2 traffic over more lines.
+    const int n_mblk = (p.M + BN - 1) / BN;
     const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
 
     if (threadIdx.x == 0) {
@@ -100,8 +102,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             uint32_t par = 1;
             bool waited_dep = false, ok = true;
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
-                const int rsb = 2 * (t % n_pairs) + (int)rank;
-                const int m0 = (t / n_pairs) * BN + 128 * (int)rank;     // this CTA's 128 tokens of the tile
+                const int rsb = 2 * (t / n_mblk) + (int)rank;
+                const int m0 = (t % n_mblk) * BN + 128 * (int)rank;      // this CTA's 128 tokens of the tile
                 const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
@@ -164,11 +166,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ------------------------------------------------------------------ dequantise
         // The MMA-issuing warp (warp 1) lives on scheduler 1 (warp id % 4); dequantise work is kept off
         // that scheduler so that the issuing thread is never queued behind ALU-heavy warps.
-        if ((warp & 3) == 1) {
-            // Spare warps 5, 9, 13, 17 of the PEER CTA relay "A slot ready" to the leader: one warp per A
+        if ((warp & 3) == 1 || warp == 23) {
+            // Spare warps 5, 9, 13, 17, 21, 23 of the PEER CTA relay "A slot ready" to the leader: one warp per A
             // slot (a waiting warp is suspended as a whole, so relay lanes of one warp would serialise),
             // one remote arrive per slot phase on the leader's afull barrier.
-            const int a = (warp - 5) >> 2;
+            const int a = warp == 23 ? 5 : (warp - 5) >> 2;
             if (rank != 0 && lane == 0 && a < NA) {
                 uint32_t apar = 0;
                 const int total_steps = n_steps * ((p.n_tiles - first_tile + tile_stride - 1) / tile_stride);
@@ -178,7 +180,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     apar ^= 1;
                 }
             }
-        } else if (warp <= 22) {                                         // 16 dequantise warps; warp 23 idles
+        } else {                                                         // 16 dequantise warps
         const DequantLane dq(warp - 2 - ((warp - 1) >> 2), lane);
         int s = 0, a = 0;
         uint32_t par = 0;
@@ -215,7 +217,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
             const int buf = j & 1;
             const uint32_t use = (uint32_t)(j >> 1);
-            const int rsb = 2 * (t % n_pairs) + (int)rank, m0 = (t / n_pairs) * BN;
+            const int rsb = 2 * (t / n_mblk) + (int)rank, m0 = (t % n_mblk) * BN;
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
             const int n = rsb * kRsbRows + quarter * 32 + lane;
