@@ -77,7 +77,9 @@ ql_status qlinear_unpack(const qlinear_desc* desc, const void* packed, int8_t* q
  *   packed_dev  device pointer, 256-byte aligned, qlinear_packed_size(desc) bytes, owned by the caller,
  *               must stay alive and unchanged until qlinear_destroy.
  *   device      CUDA device ordinal that owns packed_dev.
- * The handle owns host memory only.  Errors: QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ARCH
+ * The handle owns host memory and a small device scratch (a few MB of partial-sum slots for the streaming
+ * decode kernel, allocated here, freed by qlinear_destroy); calls on one handle must be stream-ordered.
+ * Errors: QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ARCH
  * (device is not sm_100), QL_ERR_CUDA, QL_ERR_ALLOC. */
 ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int device, qlinear_t* out);
 
@@ -104,7 +106,35 @@ ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_dev_out, void* cuda
  * identifies the wait.  Clears the condition. */
 ql_status qlinear_device_status(qlinear_t h, uint32_t* detail);
 
-/* Frees the handle's host memory.  Does not touch the packed blob.  NULL is allowed. */
+/* Decode call for callers that cannot allocate device memory.  (The paper has no counterpart: this is
+ * a deployment variant of the decode stage of Section 3.7, not a new operation.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a latency-critical serving loop
+ * whose memory was carved up front, under a memory pool that owns every byte of the device, or in a
+ * plugin that is only handed input and output buffers.  qlinear_create allocates a small device scratch
+ * for the streaming decode kernel; this call takes no handle and allocates nothing, neither on the device
+ * nor through any library: the kernel's partial-sum slots and arrival counters live in one static device
+ * array of 2,752,512 bytes (2.5 MiB of slots for at most 320 CTAs + 128 KiB of counters) that every GPU
+ * loading the library holds until the process exits.
+ *
+ *   desc, packed_dev   as for qlinear_create (the blob already in device memory, 256-byte aligned)
+ *   x_dev, y_dev, M    as for qlinear_forward, with 1 <= M <= 8 (decode only)
+ *   device             ordinal that owns the buffers; cuda_stream as for qlinear_forward
+ *
+ * Computes exactly what qlinear_forward computes for M <= 8 (same packed weights, same tolerance; the
+ * summation order differs from the default decode kernel, so results may differ in the last bit).
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and sets a kernel
+ * attribute; make that first call outside any stream capture.  Every call shares the one array, which keeps
+ * the previous call's contents: the counters are cleared on the stream before each launch, the slots are
+ * overwritten before they are read.  Two calls that overlap on the GPU (different streams, or different
+ * host threads without stream ordering between them) race on it -- serialise them.
+ * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, M outside 1..8), QL_ERR_UNSUPPORTED (descriptor
+ * not supported, more than 4096 row super-blocks i.e. N > 524288, or int4 with K not a multiple of 64),
+ * QL_ERR_ARCH, QL_ERR_CUDA. */
+ql_status qlinear_decode_static(const qlinear_desc* desc, const void* packed_dev, const void* x_dev, void* y_dev,
+                                int32_t M, int device, void* cuda_stream);
+
+/* Frees the handle's host memory and its device scratch.  Does not touch the packed blob.  NULL is allowed. */
 ql_status qlinear_destroy(qlinear_t h);
 
 /* Static, NUL-terminated description of a status code. */

@@ -21,7 +21,7 @@ QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
 
 EXPORTS = (
     "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward",
-    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_destroy",
+    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version",
 )
 
@@ -60,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_debug_unpack_device.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.qlinear_device_status.restype = ctypes.c_int
+    lib.qlinear_decode_static.argtypes = [dp, vp, vp, vp, i32, ctypes.c_int, vp]
+    lib.qlinear_decode_static.restype = ctypes.c_int
     lib.qlinear_destroy.argtypes = [vp]
     lib.qlinear_destroy.restype = ctypes.c_int
     lib.qlinear_status_string.argtypes = [ctypes.c_int]
@@ -134,6 +136,19 @@ def _stream_ptr(stream) -> ctypes.c_void_p:
     if stream is None:
         stream = torch.cuda.current_stream()
     return ctypes.c_void_p(stream.cuda_stream)
+
+
+def qlinear_decode_static(desc: Desc, packed, x, out=None, stream=None):
+    """Decode (M <= 8) without a handle and without any allocation inside the library: the caller passes the
+    packed device tensor, x and (optionally) the output tensor; see include/qlinear.h."""
+    import torch
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, desc.N), dtype=torch.float16, device=x.device)
+    _check(lib.qlinear_decode_static(ctypes.byref(desc.c()), ctypes.c_void_p(packed.data_ptr()),
+                                     ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(out.data_ptr()), M,
+                                     x.device.index or 0, _stream_ptr(stream)), "qlinear_decode_static")
+    return out
 
 
 class QLinear:

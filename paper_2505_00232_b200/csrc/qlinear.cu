@@ -7,6 +7,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/qlinear.h"
@@ -324,6 +325,117 @@ extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, voi
     else
         debug_unpack_kernel<8><<<grid, 256, 0, st>>>(h->blob + L.body_offset, q_out, L.N, L.K, L.n_kc, L.block_bytes);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+
+// ---------------------------------------------------------------------------------------------------
+// qlinear_decode_static: the streaming decode kernel for callers that cannot allocate device memory
+// (see include/qlinear.h).  Its partial-sum slots and counters live in one file-scope device array.
+namespace {
+
+constexpr int kStaticMaxCtas = 320;                 // CTAs of the persistent grid (2 per SM on a 148-SM part)
+constexpr int kStaticMaxRsb = 4096;                 // row super-blocks, i.e. N <= 524288
+constexpr size_t kStaticPartialBytes = (size_t)kStaticMaxCtas * 2 * kStreamPartialFloats * sizeof(float);   // 2.5 MiB
+constexpr size_t kStaticCounterBytes = (size_t)kStaticMaxRsb * 8 * sizeof(unsigned int);                    // 128 KiB
+constexpr int kStaticStages = 8;
+
+// Every GPU that loads the library holds this array until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticPartialBytes + kStaticCounterBytes];
+
+struct StaticDevice {
+    bool ready = false;
+    unsigned char* base = nullptr;                  // device address of g_static_scratch on this device
+    int sms = 0;
+};
+StaticDevice g_static_dev[64];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: the array's name is only a host-side stand-in, the address a
+// kernel may use comes from cudaGetSymbolAddress.
+ql_status static_setup(int device, StaticDevice** out)
+{
+    if (device < 0 || device >= 64) return QL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice& d = g_static_dev[device];
+    if (!d.ready) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+            cudaGetLastError();
+            return QL_ERR_CUDA;
+        }
+        if (major != 10) return QL_ERR_ARCH;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return QL_ERR_CUDA;
+        }
+        d.base = static_cast<unsigned char*>(ptr);
+        d.ready = true;
+    }
+    *out = &d;
+    return QL_OK;
+}
+
+template <int BITS, bool GROUPED>
+cudaError_t launch_stream_static(const StreamParams& prm, cudaStream_t st, int device)
+{
+    static bool attr_set[64] = {};
+    auto kern = gemv_stream_kernel<BITS, GROUPED, kStaticStages>;
+    const size_t smem = (size_t)kStaticStages * StreamStage<BITS>::kBytes;
+    if (!attr_set[device]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_set[device] = true;
+    }
+    return launch(kern, prm, dim3(prm.P), dim3(kStreamThreads), smem, st, 1, false);
+}
+
+}  // namespace
+
+extern "C" ql_status qlinear_decode_static(const qlinear_desc* d, const void* packed_dev, const void* x, void* y, int32_t M,
+                                           int device, void* stream)
+{
+    if (!d || !packed_dev || !x || !y) return QL_ERR_INVALID_ARG;
+    if (M < 1 || M > 8) return QL_ERR_INVALID_ARG;                       // decode kernel only
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(packed_dev) % 256) return QL_ERR_INVALID_ARG;
+    Layout L;
+    if (!make_layout(d->N, d->K, d->bits, d->group, &L)) return QL_ERR_UNSUPPORTED;
+    if (L.n_rsb > kStaticMaxRsb) return QL_ERR_UNSUPPORTED;              // beyond the static counters
+    if (L.bits == 4 && (L.K % 64)) return QL_ERR_UNSUPPORTED;            // the streaming kernel reads whole 64-k slices
+    DeviceGuard guard(device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    StaticDevice* dev = nullptr;
+    ql_status sst = static_setup(device, &dev);
+    if (sst != QL_OK) return sst;
+
+    const uint8_t* blob = static_cast<const uint8_t*>(packed_dev);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    StreamParams prm{};
+    prm.body = blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(blob + L.chan_scale_offset);
+    prm.x = static_cast<const __half*>(x);
+    prm.y = static_cast<__half*>(y);
+    prm.scratch = reinterpret_cast<float*>(dev->base);
+    prm.counters = reinterpret_cast<unsigned int*>(dev->base + kStaticPartialBytes);
+    prm.M = M; prm.N = L.N; prm.K = L.K;
+    prm.n_rsb = L.n_rsb; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
+    const int64_t B = (int64_t)L.n_rsb * L.n_kc;
+    prm.P = (int)std::min<int64_t>(B, std::min(kStaticMaxCtas, 2 * dev->sms));
+    prm.stages = kStaticStages;
+    // The array keeps whatever the last call left: the counters must start at zero (they do after a call
+    // that ran to completion; this also covers one that did not).
+    if (cudaMemsetAsync(prm.counters, 0, (size_t)L.n_rsb * 8 * sizeof(unsigned int), st) != cudaSuccess) {
+        cudaGetLastError();
+        return QL_ERR_CUDA;
+    }
+    cudaError_t e;
+    if (L.bits == 8) e = launch_stream_static<8, false>(prm, st, device);
+    else if (L.grouped) e = launch_stream_static<4, true>(prm, st, device);
+    else e = launch_stream_static<4, false>(prm, st, device);
+    if (e != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
+    return QL_OK;
 }
 
 extern "C" ql_status qlinear_device_status(qlinear_t h, uint32_t* detail)
