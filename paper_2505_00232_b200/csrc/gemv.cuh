@@ -59,7 +59,7 @@ __device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], 
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <int BITS, bool GROUPED>
+template <int BITS, bool GROUPED, bool XDIRECT>
 __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -117,8 +117,9 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // Stage this CTA's K range of x (zero beyond K) in shared memory.
-    {
+    // Stage this CTA's K range of x (zero beyond K) in shared memory -- or, in the direct form, read the
+    // x fragments straight from global memory (they stay in L1: every row-block reuses the same slice).
+    if (!XDIRECT) {
         const int span = k_cta1 - k_cta0;                                // multiple of 32
         const int vec_per_tok = span >> 3;
         for (int i = threadIdx.x; i < p.M * vec_per_tok; i += kGemvThreads) {
@@ -128,67 +129,93 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             if (k < p.K) val = *reinterpret_cast<const uint4*>(p.x + (int64_t)m * p.K + k);
             *reinterpret_cast<uint4*>(xs + m * p.x_stride + v * 8) = val;
         }
+        __syncthreads();
     }
-    __syncthreads();
 
     float total[4] = {0.f, 0.f, 0.f, 0.f};
     // Lanes whose token column does not exist (g >= M) read the last real token: MMA columns are
     // independent and those columns are never stored.
-    const __half* xpass = xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
+    const __half* xpass = XDIRECT ? p.x + (int64_t)min(g, p.M - 1) * p.K + 8 * c + kc0 * CHUNK_K
+                                  : xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
+    const __half* xend = p.x + (int64_t)(min(g, p.M - 1) + 1) * p.K;     // direct form: end of this token's row
+    auto load_x = [&](const __half* ptr) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (!XDIRECT) v = *reinterpret_cast<const uint4*>(ptr);
+        else if (ptr < xend) asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
+        return v;
+    };
     const unsigned char* wslot = ring + lane * 16;
     int sflip = 0;                                                       // scale buffer of the current pass
 
+    // one chunk: unpack in registers, feed the tensor core, apply the group scales in fp32
+    auto chunk_math = [&](const uint4& w, const uint2& sc, const __half* xk) {
+        uint32_t a[4];
+        if (BITS == 4) {
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint4 xv = load_x(xk + 32 * h);
+                if (GROUPED) {
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    unpack_int4_word(ww[2 * h], a);
+                    mma_16816_pure(acc, a, xv.x, xv.y);
+                    unpack_int4_word(ww[2 * h + 1], a);
+                    mma_16816_pure(acc, a, xv.z, xv.w);
+                    const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);          // row g:   G0, G1
+                    const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);          // row g+8: G0, G1
+                    const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
+                    const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
+                    total[0] = fmaf(sg, acc[0], total[0]);
+                    total[1] = fmaf(sg, acc[1], total[1]);
+                    total[2] = fmaf(sg8, acc[2], total[2]);
+                    total[3] = fmaf(sg8, acc[3], total[3]);
+                } else {
+                    unpack_int4_word(ww[2 * h], a);
+                    mma_16816_pure(total, a, xv.x, xv.y);
+                    unpack_int4_word(ww[2 * h + 1], a);
+                    mma_16816_pure(total, a, xv.z, xv.w);
+                }
+            }
+        } else {
+            const uint4 xv = load_x(xk);
+            unpack_int8_words(w.x, w.y, a);
+            mma_16816_pure(total, a, xv.x, xv.y);
+            unpack_int8_words(w.z, w.w, a);
+            mma_16816_pure(total, a, xv.z, xv.w);
+        }
+    };
+
+    // Two chunks per iteration: both are read into registers and their slots refilled before the math, so
+    // the two independent unpack/MMA chains interleave.
     for (int kc = kc0; kc < kc1; kc += kGemvRing) {
 #pragma unroll
-        for (int d = 0; d < kGemvRing; ++d) {
+        for (int d = 0; d < kGemvRing; d += 2) {
             if (kc + d >= kc1) break;
-            asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 1) : "memory");
+            const bool two = kc + d + 1 < kc1;
+            asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 2) : "memory");
             if (GROUPED && d == 0) {
                 __syncwarp();                                            // scales of this pass visible; last pass's reads done
                 copy16(sbuf_u32 + (sflip ^ 1) * 512, ssrc, kc + kGemvRing + (lane >> 2) < kc1);
                 ssrc += pass_bytes;
             }
-            const uint4 w = *reinterpret_cast<const uint4*>(wslot + d * 512);
-            uint2 sc = make_uint2(0, 0);
-            if (GROUPED) sc = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + d * 64 + g * 8);
-            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slot just read
+            const uint4 w0 = *reinterpret_cast<const uint4*>(wslot + d * 512);
+            const uint4 w1 = *reinterpret_cast<const uint4*>(wslot + (d + 1) * 512);
+            uint2 sc0 = make_uint2(0, 0), sc1 = make_uint2(0, 0);
+            if (GROUPED) {
+                sc0 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + d * 64 + g * 8);
+                sc1 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + (d + 1) * 64 + g * 8);
+            }
+            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slots just read
             commit();
-            wsrc += p.block_bytes;
-
+            copy16(ring_u32 + (d + 1) * 512, wsrc + p.block_bytes, kc + d + 1 + kGemvRing < kc1);
+            commit();
+            wsrc += 2 * (int64_t)p.block_bytes;
             const __half* xk = xpass + d * CHUNK_K;
-            uint32_t a[4];
-            if (BITS == 4) {
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint4 xv = *reinterpret_cast<const uint4*>(xk + 32 * h);
-                    if (GROUPED) {
-                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                        unpack_int4_word(ww[2 * h], a);
-                        mma_16816_pure(acc, a, xv.x, xv.y);
-                        unpack_int4_word(ww[2 * h + 1], a);
-                        mma_16816_pure(acc, a, xv.z, xv.w);
-                        const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);      // row g:   G0, G1
-                        const __half2 s_hi = *reinterpret_cast<const __half2*>(&sc.y);      // row g+8: G0, G1
-                        const float sg = h == 0 ? __low2float(s_lo) : __high2float(s_lo);
-                        const float sg8 = h == 0 ? __low2float(s_hi) : __high2float(s_hi);
-                        total[0] = fmaf(sg, acc[0], total[0]);
-                        total[1] = fmaf(sg, acc[1], total[1]);
-                        total[2] = fmaf(sg8, acc[2], total[2]);
-                        total[3] = fmaf(sg8, acc[3], total[3]);
-                    } else {
-                        unpack_int4_word(ww[2 * h], a);
-                        mma_16816_pure(total, a, xv.x, xv.y);
-                        unpack_int4_word(ww[2 * h + 1], a);
-                        mma_16816_pure(total, a, xv.z, xv.w);
-                    }
-                }
+            if (two) {
+                chunk_math(w0, sc0, xk);
+                chunk_math(w1, sc1, xk + CHUNK_K);
             } else {
-                const uint4 xv = *reinterpret_cast<const uint4*>(xk);
-                unpack_int8_words(w.x, w.y, a);
-                mma_16816_pure(total, a, xv.x, xv.y);
-                unpack_int8_words(w.z, w.w, a);
-                mma_16816_pure(total, a, xv.z, xv.w);
+                chunk_math(w0, sc0, xk);
             }
         }
         xpass += kGemvRing * CHUNK_K;

@@ -70,7 +70,7 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             if ((ks - 1) * cps >= L.n_kc && ks > 1) continue;               // would leave a slice empty
             const int span = std::min(ks_cta * cps, L.n_kc) * L.chunk_k;
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
-            const int x_bytes = ((M * x_stride * 2 + 127) / 128) * 128;
+            const int x_bytes = env_int("QLINEAR_GEMV_XDIRECT", 1) ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
@@ -113,17 +113,24 @@ cudaError_t launch(Kern kern, const Params& prm, dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
-template <int BITS, bool GROUPED>
-cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
+template <int BITS, bool GROUPED, bool XDIRECT>
+cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
 {
     static bool attr_set[64] = {};
-    auto kern = gemv_kernel<BITS, GROUPED>;
+    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT>;
     if (h->device >= 0 && h->device < 64 && !attr_set[h->device]) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvMaxSmem);
         if (e != cudaSuccess) return e;
         attr_set[h->device] = true;
     }
     return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
+}
+
+template <int BITS, bool GROUPED>
+cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
+{
+    return prm.x_bytes == 0 ? launch_gemv_x<BITS, GROUPED, true>(h, prm, pl, st)
+                            : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
 }
 
 ql_status forward_gemv(qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
