@@ -144,6 +144,38 @@ class LayerSet:
             if only is None or li in only:
                 self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
 
+    _STAGE = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}
+
+    def step_branched(self, cp):
+        """One pass with the data flow of a transformer layer: q, k, v read the same input and run as
+        parallel branches (three streams), then o; gate and up likewise, then down.  Same seven calls."""
+        torch = self.torch
+        main = torch.cuda.current_stream()
+        if not hasattr(self, "_side"):
+            self._side = [torch.cuda.Stream(), torch.cuda.Stream()]
+        groups, prev = [], None
+        for li, l in enumerate(self.layers):
+            st = self._STAGE.get(l.name, 100 + li)
+            if st != prev:
+                groups.append([])
+                prev = st
+            groups[-1].append(li)
+        for grp in groups:
+            fork = torch.cuda.Event()
+            fork.record(main)
+            joins = []
+            for j, li in enumerate(grp):
+                stream = main if j == 0 else self._side[(j - 1) % 2]
+                if j:
+                    stream.wait_event(fork)
+                self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M, stream)
+                if j:
+                    ev = torch.cuda.Event()
+                    ev.record(stream)
+                    joins.append(ev)
+            for ev in joins:
+                main.wait_event(ev)
+
     def step_e2e(self, cp):
         """Host buffers in, host buffers out: H2D of every x, the forwards, D2H of every y."""
         for li in range(len(self.layers)):
@@ -274,11 +306,12 @@ def run_reference(args, workload, M):
 
 
 # ------------------------------------------------------------------------------------ GPU legs
-def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index):
+def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, branches=False):
     """Times `steps` passes over the layer set; returns dict with ms_per_step, clocks, launches."""
     copies = ls.copies
     if use_graph:
-        graph = capture_graph(torch, lambda i: ls.step(i % copies), copies)
+        step_fn = ls.step_branched if branches else ls.step
+        graph = capture_graph(torch, lambda i: step_fn(i % copies), copies)
         n_replays = max(1, steps // copies)
         steps = n_replays * copies
         for _ in range(max(1, warmup // copies)):
@@ -321,6 +354,9 @@ def main():
     ap.add_argument("--M", type=int, default=0, help="tokens (default: the workload's first M)")
     ap.add_argument("--copies", type=int, default=0, help="weight copies rotated (default: enough for 3x L2, >= 4)")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA-graph replay")
+    ap.add_argument("--no-branches", action="store_true",
+                    help="decode graph: launch the seven layers strictly one after another (default: q/k/v and "
+                         "gate/up as parallel graph branches, the data flow of a transformer layer)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill sub-measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill-steps", type=int, default=20)
@@ -361,7 +397,8 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local))
+    branches = use_graph and not args.no_branches
+    res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local), branches)
     if world > 1:
         dist.barrier()
         res["ms"] = max_over_ranks(res["ms"], device)
@@ -420,7 +457,8 @@ def main():
         "config": {"workload": workload.name, "M": M, "layers": [f"{l.name}:{l.N}x{l.K}:int{l.bits}" for l in workload.layers],
                    "weight_copies": copies, "weight_bytes_per_step": ls.weight_bytes,
                    "l2": f"{copies} weight copies ({copies * layer_bytes / 1e6:.0f} MB) rotated per step; no flush",
-                   "launch": "cuda graph + programmatic dependent launch" if use_graph else "stream launches",
+                   "launch": ("cuda graph + programmatic dependent launch" + (", q/k/v and gate/up as parallel branches" if branches else ""))
+                             if use_graph else "stream launches",
                    "parallelism": "replicas only" if world > 1 else "single gpu"},
         "clocks": res["clocks"], "gpu_launches": res["launches"],
         "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": ls.h2d_bytes, "d2h_bytes_per_step": ls.d2h_bytes,

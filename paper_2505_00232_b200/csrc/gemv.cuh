@@ -38,6 +38,7 @@ struct GemvParams {
     int32_t n_kc;                        // chunks along K
     int32_t block_bytes;
     int32_t ks_cta;                      // K slices handled inside one CTA: 1, 2, 4 or 8
+    int32_t ks_cta_log2;
     int32_t cl;                          // CTAs per cluster along K (1 = no cluster)
     int32_t cps;                         // chunks per slice
     int32_t x_stride;                    // halves between tokens in the shared x slab
@@ -71,11 +72,15 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     const int g = lane >> 2, c = lane & 3;
     constexpr int CHUNK_K = BITS == 4 ? 64 : 32;
 
-    const int crank = p.cl > 1 ? (int)(blockIdx.x % p.cl) : 0;
-    const int rb_group = p.cl > 1 ? (int)(blockIdx.x / p.cl) : (int)blockIdx.x;
-    const int rb_per_cta = kGemvWarps / p.ks_cta;
-    const int ks_local = warp % p.ks_cta;
-    const int rb = rb_group * rb_per_cta + warp / p.ks_cta;
+    // No integer division on the way in: ks_cta is a power of two, and the position inside the cluster
+    // comes from the special registers (without a cluster launch they read rank 0, cluster id = block id).
+    uint32_t crank_u, rb_group_u;
+    asm("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank_u));
+    asm("mov.u32 %0, %%clusterid.x;" : "=r"(rb_group_u));
+    const int crank = (int)crank_u, rb_group = (int)rb_group_u;
+    const int rb_per_cta = kGemvWarps >> p.ks_cta_log2;
+    const int ks_local = warp & (p.ks_cta - 1);
+    const int rb = rb_group * rb_per_cta + (warp >> p.ks_cta_log2);
     const bool rb_live = rb < p.n_rb;
     const int ks = crank * p.ks_cta + ks_local;
     const int kc0 = min(ks * p.cps, p.n_kc);

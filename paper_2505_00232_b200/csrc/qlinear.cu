@@ -146,7 +146,7 @@ ql_status forward_gemv(qlinear_s* h, const void* x, void* y, int M, cudaStream_t
     prm.n_rb = (L.N + kRbRows - 1) / kRbRows;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
-    prm.ks_cta = pl.ks_cta; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
+    prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
     cudaError_t e;
     if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st);
     else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st);
