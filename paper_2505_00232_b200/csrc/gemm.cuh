@@ -44,7 +44,10 @@ struct GemmParams {
     int32_t M, N, K;
     int32_t n_kc, block_bytes;
     int32_t n_ksteps;
-    int32_t n_rsb, n_tiles;                  // tiles = n_rsb x ceil(M / BN); tile t -> (t % n_rsb, t / n_rsb)
+    int32_t n_rsb, n_tiles;                  // work units of the grid (pair kernel: tiles x split)
+    int32_t split;                           // pair kernel: K split of every tile (1 = none)
+    float* scratch;                          // pair kernel, split > 1: fp32 partial tiles [tile][part][rank][256][128]
+    unsigned int* counters;                  // pair kernel, split > 1: arrivals per (tile, rank, quarter), zero between launches
 };
 
 struct GemmPlan {

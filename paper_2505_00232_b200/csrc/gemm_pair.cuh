@@ -64,7 +64,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                             // 0 = leader
-    const int n_steps = p.n_ksteps;
+    // A work unit is one K part of one tile: unit t -> tile t / KS, part t % KS; with KS > 1 the parts of a
+    // tile run on different clusters at the same time and are added up by the last one to finish.
+    const int KS = p.split;
+    const int n_steps = p.n_ksteps / KS;                                  // k-steps per unit
     // Tile t = (row-super-block pair t / n_mblk, token block t % n_mblk): clusters that run side by side share
     // weight blocks and read different x tiles, which spreads the L2 traffic over more lines.
     const int n_mblk = (p.M + BN - 1) / BN;
@@ -102,13 +105,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             uint32_t par = 1;
             bool waited_dep = false, ok = true;
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
-                const int rsb = 2 * (t / n_mblk) + (int)rank;
-                const int m0 = (t % n_mblk) * BN + 128 * (int)rank;      // this CTA's 128 tokens of the tile
+                const int tile = t / KS, step0 = (t - tile * KS) * n_steps;
+                const int rsb = 2 * (tile / n_mblk) + (int)rank;
+                const int m0 = (tile % n_mblk) * BN + 128 * (int)rank;   // this CTA's 128 tokens of the tile
                 const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
                     QL_GTRACE(0, issued);
-                    const int kc = it * CHUNKS;
+                    const int kc = (step0 + it) * CHUNKS;
                     const int nblk = min(CHUNKS, p.n_kc - kc);
                     const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
                     mbar_expect_tx(full_bar(s), wbytes + S::kXBytes);
@@ -117,7 +121,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         waited_dep = true;
                     }
-                    tma_load_2d(xs_addr(s), &x_map, it * kGemmKStep, m0, full_bar(s));
+                    tma_load_2d(xs_addr(s), &x_map, (step0 + it) * kGemmKStep, m0, full_bar(s));
                     ++issued;
                     if (++s == NS) { s = 0; par ^= 1; }
                 }
@@ -217,7 +221,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
             const int buf = j & 1;
             const uint32_t use = (uint32_t)(j >> 1);
-            const int rsb = 2 * (t / n_mblk) + (int)rank, m0 = (t % n_mblk) * BN;
+            const int tile = t / KS, part = t - tile * KS;
+            const int rsb = 2 * (tile / n_mblk) + (int)rank, m0 = (tile % n_mblk) * BN;
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
             const int n = rsb * kRsbRows + quarter * 32 + lane;
@@ -225,21 +230,78 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             if (!GROUPED && n < p.N) scale = __half2float(p.chan_scales[n]);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
             __half* yrow = p.y + (int64_t)m0 * p.N + n;
-            const int m_left = p.M - m0;
+            const int m_left = min(BN, p.M - m0);
+            if (KS == 1) {
 #pragma unroll 1
-            for (int cc = 0; cc < BN; cc += 16) {
-                if (cc >= m_left) break;
-                uint32_t r[16];
-                tmem_ld16(taddr + (uint32_t)cc, r);
-                if (n < p.N) {
+                for (int cc = 0; cc < m_left; cc += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)cc, r);
+                    if (n < p.N) {
 #pragma unroll
-                    for (int q = 0; q < 16; ++q)
-                        if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(__uint_as_float(r[q]) * scale);
+                        for (int q = 0; q < 16; ++q)
+                            if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(__uint_as_float(r[q]) * scale);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0);
+            } else {
+                // K-split tile: park this part's fp32 accumulator in scratch ([token][channel], so a warp
+                // writes 128 contiguous bytes per token), free the accumulator, then count arrivals; the
+                // last part to arrive adds all parts in part order (fixed order, no float atomics) and stores y.
+                float* slab = p.scratch + (((int64_t)tile * KS + part) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
+#pragma unroll 1
+                for (int cc = 0; cc < m_left; cc += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(taddr + (uint32_t)cc, r);
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) __stcg(slab + (cc + q) * 128, __uint_as_float(r[q]));
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0);
+                __threadfence();
+                __syncwarp();
+                unsigned int old = 0;
+                unsigned int* cnt = p.counters + (tile * 2 + rank) * 4 + quarter;
+                if (lane == 0) old = atomicAdd(cnt, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if ((int)old == KS - 1) {
+                    __threadfence();
+                    const float* first = p.scratch + (((int64_t)tile * KS) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
+                    // all loads of a 16-token batch (every part) are issued before the ordered sum, so that
+                    // the L2 round trips overlap
+#pragma unroll 1
+                    for (int cc = 0; cc < m_left; cc += 16) {
+                        float acc[16];
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) acc[q] = __ldcg(first + (cc + q) * 128);
+                        if (KS == 2) {
+                            float v[16];
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) v[q] = __ldcg(first + (int64_t)2 * (BN * 128) + (cc + q) * 128);
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) acc[q] += v[q];
+                        } else {
+                            float v1[16], v2[16], v3[16];
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) {
+                                v1[q] = __ldcg(first + (int64_t)2 * (BN * 128) + (cc + q) * 128);
+                                v2[q] = __ldcg(first + (int64_t)4 * (BN * 128) + (cc + q) * 128);
+                                v3[q] = __ldcg(first + (int64_t)6 * (BN * 128) + (cc + q) * 128);
+                            }
+#pragma unroll
+                            for (int q = 0; q < 16; ++q) acc[q] = ((acc[q] + v1[q]) + v2[q]) + v3[q];
+                        }
+                        if (n < p.N) {
+#pragma unroll
+                            for (int q = 0; q < 16; ++q)
+                                if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(acc[q] * scale);
+                        }
+                    }
+                    if (lane == 0) *cnt = 0;                             // ready for the next launch
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0);
         }
     }
 
@@ -252,9 +314,28 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     }
 }
 
+// K split of every tile: used when there are fewer tiles than half the clusters, so that the whole GPU works
+// on skinny layers.  Units never exceed the cluster count, which bounds the scratch (see gemm_pair_scratch_bytes).
+inline int gemm_pair_split(int tiles, int n_ksteps, int num_sms, bool have_scratch)
+{
+    if (!have_scratch) return 1;
+    const char* f = std::getenv("QLINEAR_GEMM_SPLIT");
+    const int clusters = num_sms / 2;
+    int split = 1;
+    if (f && *f && std::atoi(f) > 0) split = std::atoi(f);
+    else if (tiles * 4 <= clusters) split = 4;
+    else if (tiles * 2 <= clusters) split = 2;
+    while (split > 1 && (n_ksteps % split || n_ksteps / split < 8 || tiles * split > clusters)) split >>= 1;
+    return split == 3 ? 2 : split;                                       // the kernel adds 2 or 4 parts
+}
+inline size_t gemm_pair_scratch_bytes(int num_sms) { return (size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float); }
+inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 8; }
+// A layer can only ever be split if it has few row-super-block pairs.
+inline bool gemm_pair_may_split(const Layout& L, int num_sms) { return (L.n_rsb % 2) == 0 && (L.n_rsb / 2) * 2 <= num_sms / 2; }
+
 template <int BITS, bool GROUPED>
 ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device,
-                           bool pdl, int num_sms)
+                           bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
     using S = GemmPairSmem<BITS>;
     EncodeTiledFn enc = get_encode_tiled();
@@ -285,7 +366,11 @@ ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, 
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
     prm.n_rsb = L.n_rsb;
-    prm.n_tiles = (L.n_rsb / 2) * ((M + 255) / 256);
+    const int tiles = (L.n_rsb / 2) * ((M + 255) / 256);
+    prm.split = gemm_pair_split(tiles, prm.n_ksteps, num_sms, scratch != nullptr);
+    prm.scratch = scratch;
+    prm.counters = counters;
+    prm.n_tiles = tiles * prm.split;                                     // work units
     const int n_clusters = prm.n_tiles < num_sms / 2 ? prm.n_tiles : num_sms / 2;
 
     cudaLaunchConfig_t cfg{};
@@ -318,11 +403,11 @@ inline bool gemm_pair_applicable(const Layout& L, int M)
 }
 
 inline ql_status gemm_pair_forward(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st,
-                                   int device, bool pdl, int num_sms)
+                                   int device, bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
-    if (L.bits == 8) return gemm_pair_launch<8, false>(L, blob, x, y, M, st, device, pdl, num_sms);
-    if (L.grouped) return gemm_pair_launch<4, true>(L, blob, x, y, M, st, device, pdl, num_sms);
-    return gemm_pair_launch<4, false>(L, blob, x, y, M, st, device, pdl, num_sms);
+    if (L.bits == 8) return gemm_pair_launch<8, false>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    if (L.grouped) return gemm_pair_launch<4, true>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    return gemm_pair_launch<4, false>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
 }
 
 }  // namespace ql

@@ -44,6 +44,9 @@ struct qlinear_s {
     int stream_P, stream_stages;
     float* stream_scratch;     // device, owned: [P][2][1024] fp32 partial sums
     unsigned int* stream_counters;   // device, owned: [n_rsb][8], zero between launches
+    // prefill pair kernel, K-split of skinny layers
+    float* gemm_scratch;             // device, owned (nullptr if the layer can never be split)
+    unsigned int* gemm_counters;     // device, owned, zero between launches
 };
 
 namespace {
@@ -295,6 +298,16 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
         if (cudaMalloc(&h->stream_counters, cbytes) != cudaSuccess || cudaMemset(h->stream_counters, 0, cbytes) != cudaSuccess) {
             cudaGetLastError(); cudaFree(h->stream_scratch); cudaFree(h->stream_counters); delete h; return QL_ERR_CUDA;
         }
+        if (gemm_pair_may_split(L, sms)) {
+            const size_t cb = gemm_pair_counter_count(sms) * sizeof(unsigned int);
+            if (cudaMalloc(&h->gemm_scratch, gemm_pair_scratch_bytes(sms)) != cudaSuccess ||
+                cudaMalloc(&h->gemm_counters, cb) != cudaSuccess || cudaMemset(h->gemm_counters, 0, cb) != cudaSuccess) {
+                cudaGetLastError();
+                cudaFree(h->stream_scratch); cudaFree(h->stream_counters); cudaFree(h->gemm_scratch); cudaFree(h->gemm_counters);
+                delete h;
+                return QL_ERR_CUDA;
+            }
+        }
     }
     *out = h;
     return QL_OK;
@@ -315,7 +328,8 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(h, x, y, M, st);
-    if (gemm_pair_applicable(h->L, M)) return gemm_pair_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
+    if (gemm_pair_applicable(h->L, M))
+        return gemm_pair_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms, h->gemm_scratch, h->gemm_counters);
     return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
@@ -467,6 +481,8 @@ extern "C" ql_status qlinear_destroy(qlinear_t h)
         DeviceGuard guard(h->device);
         cudaFree(h->stream_scratch);
         cudaFree(h->stream_counters);
+        cudaFree(h->gemm_scratch);
+        cudaFree(h->gemm_counters);
     }
     delete h;
     return QL_OK;

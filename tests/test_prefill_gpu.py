@@ -48,6 +48,8 @@ SMALL = [
     (127, 264, 2304, 4, 32), (128, 128, 1056, 8, 0), (129, 384, 1024, 4, 32), (300, 520, 1056, 8, 0),
     (256, 40, 256, 4, 64), (257, 16, 384, 4, 128), (512, 1000, 96, 8, 0), (1024, 256, 2304, 4, 32),
     (700, 384, 4096, 8, 0), (2048, 128, 14336, 4, 32),
+    # few tiles: the CTA-pair kernel splits K across clusters and adds the parts through scratch
+    (600, 512, 2048, 8, 0), (300, 256, 4096, 4, 32), (1024, 1024, 1024, 4, 0),
 ]
 
 
@@ -73,6 +75,16 @@ def test_one_hot_rows_return_rounded_weight_columns_bit_exact(P, torch, N, K, bi
     y = forward(P, torch, lin, x)
     want = (s[:, ks // G].astype(np.float64) * q[:, ks].astype(np.float64)).astype(np.float16).T   # [M, N]
     assert (y.view(np.uint16) == want.view(np.uint16)).all()
+
+
+def test_split_k_is_deterministic_and_counters_reset(P, torch):
+    q, s, x = rand_case(47, 600, 512, 2048, 8, 0)
+    lin = P.QLinear.from_weights(q, s, 8, 0, device="cuda:0")
+    xd = torch.from_numpy(x).cuda()
+    a = lin.forward(xd).clone()
+    for _ in range(4):
+        assert torch.equal(a, lin.forward(xd))
+    assert_parity(a.cpu().numpy(), x, q, s, 0)
 
 
 def test_zero_input_gives_positive_zero(P, torch):
