@@ -45,7 +45,8 @@ struct GemmParams {
     int32_t n_kc, block_bytes;
     int32_t n_ksteps;
     int32_t n_rsb, n_tiles;                  // work units of the grid (pair kernel: tiles x split)
-    int32_t split;                           // pair kernel: K split of every tile (1 = none)
+    int32_t split;                           // pair kernel: K parts of the tiles that are split (1 = none are)
+    int32_t n_whole;                         // pair kernel: units [0, n_whole) are whole tiles, the rest are parts
     float* scratch;                          // pair kernel, split > 1: fp32 partial tiles [tile][part][rank][256][128]
     unsigned int* counters;                  // pair kernel, split > 1: arrivals per (tile, rank, quarter), zero between launches
 };

@@ -35,6 +35,28 @@ struct GemmPairSmem {
     static constexpr int kTotal = kBarOffset + 512 + 1024;               // barriers + alignment slack
 };
 
+// Work unit t of the grid: a whole tile (t < n_whole) or one K part of a split tile.  Whole tiles fill the
+// full rounds of the persistent grid; the tiles of the last, partial round are split so that it is short.
+struct PairUnit {
+    int tile, part, parts, step0, nsteps, slab;
+};
+__device__ __forceinline__ PairUnit pair_unit(int t, const GemmParams& p)
+{
+    PairUnit u;
+    if (t < p.n_whole) {
+        u.tile = t; u.part = 0; u.parts = 1; u.step0 = 0; u.nsteps = p.n_ksteps; u.slab = 0;
+    } else {
+        const int v = t - p.n_whole;
+        u.slab = v / p.split;                                            // index among the split tiles (scratch slot)
+        u.tile = p.n_whole + u.slab;
+        u.part = v - u.slab * p.split;
+        u.parts = p.split;
+        u.nsteps = p.n_ksteps / p.split;
+        u.step0 = u.part * u.nsteps;
+    }
+    return u;
+}
+
 template <int BITS, bool GROUPED>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
@@ -64,10 +86,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();                             // 0 = leader
-    // A work unit is one K part of one tile: unit t -> tile t / KS, part t % KS; with KS > 1 the parts of a
-    // tile run on different clusters at the same time and are added up by the last one to finish.
     const int KS = p.split;
-    const int n_steps = p.n_ksteps / KS;                                  // k-steps per unit
     // Tile t = (row-super-block pair t / n_mblk, token block t % n_mblk): clusters that run side by side share
     // weight blocks and read different x tiles, which spreads the L2 traffic over more lines.
     const int n_mblk = (p.M + BN - 1) / BN;
@@ -105,7 +124,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             uint32_t par = 1;
             bool waited_dep = false, ok = true;
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
-                const int tile = t / KS, step0 = (t - tile * KS) * n_steps;
+                const PairUnit u = pair_unit(t, p);
+                const int tile = u.tile, step0 = u.step0, n_steps = u.nsteps;
                 const int rsb = 2 * (tile / n_mblk) + (int)rank;
                 const int m0 = (tile % n_mblk) * BN + 128 * (int)rank;   // this CTA's 128 tokens of the tile
                 const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
@@ -143,6 +163,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
                 const int buf = j & 1;
                 const uint32_t use = (uint32_t)(j >> 1);
+                const int n_steps = pair_unit(t, p).nsteps;
                 if (!mbar_wait(tempty_bar(buf), (use & 1) ^ 1, abort_flag, 0x800 + buf)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
@@ -150,7 +171,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     // own A tile written (implies own x half landed) and the peer's likewise
                     // 16 local dequantise warps + the peer's relay lane: both A tiles written, both x halves landed
                     if (!mbar_wait(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
-                    QL_GTRACE(5, j * n_steps + it);
+                    QL_GTRACE(5, j * p.n_ksteps + it);
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
@@ -159,7 +180,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)
                         umma_f16_pair_lo(tmem_d, a_lo + 2 * k4, b_lo + 2 * k4, idesc, 1u);
                     umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
-                    QL_GTRACE(6, j * n_steps + it);
+                    QL_GTRACE(6, j * p.n_ksteps + it);
                     if (++s == NS) s = 0;
                     if (++a == NA) { a = 0; apar ^= 1; }
                 }
@@ -177,7 +198,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             const int a = warp == 23 ? 5 : (warp - 5) >> 2;
             if (rank != 0 && lane == 0 && a < NA) {
                 uint32_t apar = 0;
-                const int total_steps = n_steps * ((p.n_tiles - first_tile + tile_stride - 1) / tile_stride);
+                int total_steps = 0;
+                for (int t = first_tile; t < p.n_tiles; t += tile_stride) total_steps += pair_unit(t, p).nsteps;
                 for (int g = a; g < total_steps; g += NA) {
                     if (!mbar_wait(afull_bar(a), apar, abort_flag, 0xA00 + a)) break;
                     mbar_arrive_remote(afull_bar(a), 0);
@@ -195,6 +217,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         bool ok = true;
         int gstep = 0;
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+            const int n_steps = pair_unit(t, p).nsteps;
             for (int it = 0; it < n_steps; ++it, ++gstep) {
                 if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
                 if (threadIdx.x == 64) QL_GTRACE(1, gstep);
@@ -221,7 +244,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
             const int buf = j & 1;
             const uint32_t use = (uint32_t)(j >> 1);
-            const int tile = t / KS, part = t - tile * KS;
+            const PairUnit u = pair_unit(t, p);
+            const int tile = u.tile, part = u.part;
             const int rsb = 2 * (tile / n_mblk) + (int)rank, m0 = (tile % n_mblk) * BN;
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
@@ -231,7 +255,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
             __half* yrow = p.y + (int64_t)m0 * p.N + n;
             const int m_left = min(BN, p.M - m0);
-            if (KS == 1) {
+            if (u.parts == 1) {
 #pragma unroll 1
                 for (int cc = 0; cc < m_left; cc += 16) {
                     uint32_t r[16];
@@ -249,7 +273,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 // K-split tile: park this part's fp32 accumulator in scratch ([token][channel], so a warp
                 // writes 128 contiguous bytes per token), free the accumulator, then count arrivals; the
                 // last part to arrive adds all parts in part order (fixed order, no float atomics) and stores y.
-                float* slab = p.scratch + (((int64_t)tile * KS + part) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
+                float* slab = p.scratch + (((int64_t)u.slab * KS + part) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
 #pragma unroll 1
                 for (int cc = 0; cc < m_left; cc += 16) {
                     uint32_t r[16];
@@ -263,12 +287,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 __threadfence();
                 __syncwarp();
                 unsigned int old = 0;
-                unsigned int* cnt = p.counters + (tile * 2 + rank) * 4 + quarter;
+                unsigned int* cnt = p.counters + (u.slab * 2 + rank) * 4 + quarter;
                 if (lane == 0) old = atomicAdd(cnt, 1u);
                 old = __shfl_sync(0xffffffffu, old, 0);
                 if ((int)old == KS - 1) {
                     __threadfence();
-                    const float* first = p.scratch + (((int64_t)tile * KS) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
+                    const float* first = p.scratch + (((int64_t)u.slab * KS) * 2 + rank) * (BN * 128) + quarter * 32 + lane;
                     // all loads of a 16-token batch (every part) are issued before the ordered sum, so that
                     // the L2 round trips overlap
 #pragma unroll 1
@@ -316,12 +340,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 
 // K split of every tile: used when there are fewer tiles than half the clusters, so that the whole GPU works
 // on skinny layers.  Units never exceed the cluster count, which bounds the scratch (see gemm_pair_scratch_bytes).
-inline int gemm_pair_split(int tiles, int n_ksteps, int num_sms, bool have_scratch)
+inline int gemm_pair_split(int tiles /* of the last, partial round */, int n_ksteps, int num_sms, bool have_scratch)
 {
     if (!have_scratch) return 1;
     const char* f = std::getenv("QLINEAR_GEMM_SPLIT");
     const int clusters = num_sms / 2;
     int split = 1;
+    if (tiles == 0) return 1;
     if (f && *f && std::atoi(f) > 0) split = std::atoi(f);
     else if (tiles * 4 <= clusters) split = 4;
     else if (tiles * 2 <= clusters) split = 2;
@@ -331,7 +356,7 @@ inline int gemm_pair_split(int tiles, int n_ksteps, int num_sms, bool have_scrat
 inline size_t gemm_pair_scratch_bytes(int num_sms) { return (size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float); }
 inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 8; }
 // A layer can only ever be split if it has few row-super-block pairs.
-inline bool gemm_pair_may_split(const Layout& L, int num_sms) { return (L.n_rsb % 2) == 0 && (L.n_rsb / 2) * 2 <= num_sms / 2; }
+inline bool gemm_pair_may_split(const Layout& L, int) { return (L.n_rsb % 2) == 0; }
 
 template <int BITS, bool GROUPED>
 ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device,
@@ -367,10 +392,16 @@ ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, 
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
     prm.n_rsb = L.n_rsb;
     const int tiles = (L.n_rsb / 2) * ((M + 255) / 256);
-    prm.split = gemm_pair_split(tiles, prm.n_ksteps, num_sms, scratch != nullptr);
+    // whole tiles fill the full rounds of the persistent grid; the tiles of the last partial round are split
+    const int clusters = num_sms / 2;
+    // (splitting the tail of a multi-round schedule was measured and does not pay: the exposed scratch
+    // reduction costs what the shorter last round saves; only single-round layers are split)
+    const int tail = tiles < clusters ? tiles : 0;
+    prm.split = gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr);
+    prm.n_whole = prm.split > 1 ? tiles - tail : tiles;
     prm.scratch = scratch;
     prm.counters = counters;
-    prm.n_tiles = tiles * prm.split;                                     // work units
+    prm.n_tiles = prm.n_whole + (tiles - prm.n_whole) * prm.split;       // work units
     const int n_clusters = prm.n_tiles < num_sms / 2 ? prm.n_tiles : num_sms / 2;
 
     cudaLaunchConfig_t cfg{};

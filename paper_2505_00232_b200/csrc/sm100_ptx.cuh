@@ -34,6 +34,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Same test without a suspend hint: returns at once, for a hot poll by a thread on the critical path.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded hot wait (polls, never suspended): lowest wake-up latency, costs issue slots while waiting.
+__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code)
+{
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = code;
+            atomicExch(&g_device_flag[0], code);
+            atomicAdd(&g_device_flag[1], 1u);
+            return false;
+        }
+    }
+}
+
 // Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.
 // SLEEP: back off between polls (for waits that are long and off the critical path, so that the issue
 // slots go to warps that have work); without it the wait wakes up as soon as the phase completes.
