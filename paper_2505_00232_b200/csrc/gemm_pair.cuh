@@ -23,13 +23,17 @@ namespace ql {
 constexpr int kPairFirstEpilogueWarp = 24;
 constexpr int kPairThreads = 28 * 32;
 
-template <int BITS>
+// TB = token blocks (of 256) per tile.  With TB = 2 every dequantised A slot feeds two MMA groups (two
+// accumulators of 256 columns fill the tensor memory, so the epilogue is no longer hidden under the next
+// tile): half the dequantise work and half the A-slot hand-offs per flop.
+template <int BITS, int TB>
 struct GemmPairSmem {
-    static constexpr int kXBytes = 128 * 128;                            // this CTA's 128 tokens x 64 k
+    static constexpr int kXBlockBytes = 128 * 128;                       // this CTA's 128 tokens x 64 k of one token block
+    static constexpr int kXBytes = TB * kXBlockBytes;
     static constexpr int kWpkStride = BITS == 4 ? 5120 : 8192;           // packed block(s) of one k-step
     static constexpr int kStageBytes = kXBytes + kWpkStride;
-    static constexpr int kStages = BITS == 4 ? 6 : 5;
-    static constexpr int kASlots = 5;                                    // one relay warp per slot (warps 5, 9, 13, 17, 21, 23)
+    static constexpr int kStages = TB == 2 ? 4 : (BITS == 4 ? 6 : 5);
+    static constexpr int kASlots = TB == 2 ? 4 : 5;                      // one relay warp per slot (spare warps 5, 9, 13, 17, 21)
     static constexpr int kAOffset = kStages * kStageBytes;
     static constexpr int kBarOffset = kAOffset + kASlots * kGemmATileBytes;
     static constexpr int kTotal = kBarOffset + 512 + 1024;               // barriers + alignment slack
@@ -57,14 +61,15 @@ __device__ __forceinline__ PairUnit pair_unit(int t, const GemmParams& p)
     return u;
 }
 
-template <int BITS, bool GROUPED>
+template <int BITS, bool GROUPED, int TB>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
-    using S = GemmPairSmem<BITS>;
+    using S = GemmPairSmem<BITS, TB>;
     constexpr int NS = S::kStages;
     constexpr int NA = S::kASlots;
-    constexpr int BN = 256;                                              // tokens per tile (128 per CTA)
+    constexpr int BN = 256;                                              // tokens per MMA (128 per CTA)
+    constexpr int TILE_N = BN * TB;                                      // tokens per tile
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -89,7 +94,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     const int KS = p.split;
     // Tile t = (row-super-block pair t / n_mblk, token block t % n_mblk): clusters that run side by side share
     // weight blocks and read different x tiles, which spreads the L2 traffic over more lines.
-    const int n_mblk = (p.M + BN - 1) / BN;
+    const int n_mblk = (p.M + TILE_N - 1) / TILE_N;
     const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
 
     if (threadIdx.x == 0) {
@@ -127,7 +132,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const PairUnit u = pair_unit(t, p);
                 const int tile = u.tile, step0 = u.step0, n_steps = u.nsteps;
                 const int rsb = 2 * (tile / n_mblk) + (int)rank;
-                const int m0 = (tile % n_mblk) * BN + 128 * (int)rank;   // this CTA's 128 tokens of the tile
+                const int m0 = (tile % n_mblk) * TILE_N + 128 * (int)rank;   // this CTA's 128 tokens of each token block
                 const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
@@ -141,7 +146,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         waited_dep = true;
                     }
-                    tma_load_2d(xs_addr(s), &x_map, (step0 + it) * kGemmKStep, m0, full_bar(s));
+#pragma unroll
+                    for (int tb = 0; tb < TB; ++tb)
+                        tma_load_2d(xs_addr(s) + tb * S::kXBlockBytes, &x_map, (step0 + it) * kGemmKStep, m0 + tb * BN, full_bar(s));
                     ++issued;
                     if (++s == NS) { s = 0; par ^= 1; }
                 }
@@ -161,8 +168,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             bool ok = true;
             int j = 0;
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
-                const int buf = j & 1;
-                const uint32_t use = (uint32_t)(j >> 1);
+                // TB = 1: two accumulators alternate; TB = 2: both are used by every tile
+                const int buf = TB == 1 ? (j & 1) : 0;
+                const uint32_t use = TB == 1 ? (uint32_t)(j >> 1) : (uint32_t)j;
                 const int n_steps = pair_unit(t, p).nsteps;
                 if (!mbar_wait(tempty_bar(buf), (use & 1) ^ 1, abort_flag, 0x800 + buf)) { ok = false; break; }
                 tc_fence_after();
@@ -175,10 +183,14 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
-                    umma_f16_pair_lo(tmem_d, a_lo, b_lo, idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)
-                        umma_f16_pair_lo(tmem_d, a_lo + 2 * k4, b_lo + 2 * k4, idesc, 1u);
+                    for (int tb = 0; tb < TB; ++tb) {
+                        const uint32_t d = tmem_d + (uint32_t)(tb * BN), bl = b_lo + (uint32_t)tb * (S::kXBlockBytes >> 4);
+                        umma_f16_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
+#pragma unroll
+                        for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)
+                            umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                    }
                     umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
                     QL_GTRACE(6, j * p.n_ksteps + it);
                     if (++s == NS) s = 0;
@@ -242,11 +254,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         bool ok = true;
         int j = 0;
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
-            const int buf = j & 1;
-            const uint32_t use = (uint32_t)(j >> 1);
+            const int buf = TB == 1 ? (j & 1) : 0;
+            const uint32_t use = TB == 1 ? (uint32_t)(j >> 1) : (uint32_t)j;
             const PairUnit u = pair_unit(t, p);
             const int tile = u.tile, part = u.part;
-            const int rsb = 2 * (tile / n_mblk) + (int)rank, m0 = (tile % n_mblk) * BN;
+            const int rsb = 2 * (tile / n_mblk) + (int)rank, m0 = (tile % n_mblk) * TILE_N;
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
             const int n = rsb * kRsbRows + quarter * 32 + lane;
@@ -254,7 +266,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             if (!GROUPED && n < p.N) scale = __half2float(p.chan_scales[n]);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
             __half* yrow = p.y + (int64_t)m0 * p.N + n;
-            const int m_left = min(BN, p.M - m0);
+            const int m_left = min(TILE_N, p.M - m0);                    // accumulator column = token m0 + column
             if (u.parts == 1) {
 #pragma unroll 1
                 for (int cc = 0; cc < m_left; cc += 16) {
@@ -358,11 +370,11 @@ inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2
 // A layer can only ever be split if it has few row-super-block pairs.
 inline bool gemm_pair_may_split(const Layout& L, int) { return (L.n_rsb % 2) == 0; }
 
-template <int BITS, bool GROUPED>
+template <int BITS, bool GROUPED, int TB>
 ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device,
                            bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
-    using S = GemmPairSmem<BITS>;
+    using S = GemmPairSmem<BITS, TB>;
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return QL_ERR_CUDA;
     CUtensorMap map;
@@ -374,7 +386,7 @@ ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, 
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return QL_ERR_CUDA;
-    auto kern = gemm_pair_kernel<BITS, GROUPED>;
+    auto kern = gemm_pair_kernel<BITS, GROUPED, TB>;
     static bool attr_set[64] = {};
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
@@ -391,13 +403,13 @@ ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, 
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
     prm.n_rsb = L.n_rsb;
-    const int tiles = (L.n_rsb / 2) * ((M + 255) / 256);
+    const int tiles = (L.n_rsb / 2) * ((M + 256 * TB - 1) / (256 * TB));
     // whole tiles fill the full rounds of the persistent grid; the tiles of the last partial round are split
     const int clusters = num_sms / 2;
     // (splitting the tail of a multi-round schedule was measured and does not pay: the exposed scratch
     // reduction costs what the shorter last round saves; only single-round layers are split)
     const int tail = tiles < clusters ? tiles : 0;
-    prm.split = gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr);
+    prm.split = TB == 1 ? gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr) : 1;
     prm.n_whole = prm.split > 1 ? tiles - tail : tiles;
     prm.scratch = scratch;
     prm.counters = counters;
@@ -436,9 +448,25 @@ inline bool gemm_pair_applicable(const Layout& L, int M)
 inline ql_status gemm_pair_forward(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st,
                                    int device, bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
-    if (L.bits == 8) return gemm_pair_launch<8, false>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-    if (L.grouped) return gemm_pair_launch<4, true>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-    return gemm_pair_launch<4, false>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    // Token blocks per tile: a step of a 512-token tile costs two steps of a 256-token tile (the kernel is
+    // bound by the tensor pipe and its operand traffic, not by dequantisation), so the wider tile only pays
+    // where it saves rounds of the persistent grid.
+    const char* f = std::getenv("QLINEAR_GEMM_TB");
+    int tb = (f && *f) ? std::atoi(f) : 0;
+    if (tb == 0) {
+        const int clusters = num_sms / 2, pairs = L.n_rsb / 2;
+        const int tiles1 = pairs * ((M + 255) / 256), tiles2 = pairs * ((M + 511) / 512);
+        const int rounds1 = (tiles1 + clusters - 1) / clusters, rounds2 = (tiles2 + clusters - 1) / clusters;
+        tb = (tiles1 >= clusters && 2 * rounds2 <= rounds1) ? 2 : 1;
+    }
+    if (tb == 2 && M > 256) {
+        if (L.bits == 8) return gemm_pair_launch<8, false, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+        if (L.grouped) return gemm_pair_launch<4, true, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+        return gemm_pair_launch<4, false, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    }
+    if (L.bits == 8) return gemm_pair_launch<8, false, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    if (L.grouped) return gemm_pair_launch<4, true, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    return gemm_pair_launch<4, false, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
 }
 
 }  // namespace ql
