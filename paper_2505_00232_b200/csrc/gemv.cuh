@@ -153,13 +153,13 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     int sflip = 0;                                                       // scale buffer of the current pass
 
     // one chunk: unpack in registers, feed the tensor core, apply the group scales in fp32
-    auto chunk_math = [&](const uint4& w, const uint2& sc, const __half* xk) {
+    auto chunk_math = [&](const uint4& w, const uint2& sc, const uint4& xa, const uint4& xb) {
         uint32_t a[4];
         if (BITS == 4) {
             const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const uint4 xv = load_x(xk + 32 * h);
+                const uint4 xv = h == 0 ? xa : xb;
                 if (GROUPED) {
                     float acc[4] = {0.f, 0.f, 0.f, 0.f};
                     unpack_int4_word(ww[2 * h], a);
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
                 }
             }
         } else {
-            const uint4 xv = load_x(xk);
+            const uint4 xv = xa;
             unpack_int8_words(w.x, w.y, a);
             mma_16816_pure(total, a, xv.x, xv.y);
             unpack_int8_words(w.z, w.w, a);
@@ -197,6 +197,11 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
         for (int d = 0; d < kGemvRing; d += 2) {
             if (kc + d >= kc1) break;
             const bool two = kc + d + 1 < kc1;
+            // x fragments first: their latency (L1 / shared) runs under the wait for the weights
+            const __half* xk = xpass + d * CHUNK_K;
+            const uint4 x00 = load_x(xk), x10 = load_x(xk + CHUNK_K);
+            uint4 x01 = x00, x11 = x10;
+            if (BITS == 4) { x01 = load_x(xk + 32); x11 = load_x(xk + CHUNK_K + 32); }
             asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 2) : "memory");
             if (GROUPED && d == 0) {
                 __syncwarp();                                            // scales of this pass visible; last pass's reads done
@@ -215,12 +220,11 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             copy16(ring_u32 + (d + 1) * 512, wsrc + p.block_bytes, kc + d + 1 + kGemvRing < kc1);
             commit();
             wsrc += 2 * (int64_t)p.block_bytes;
-            const __half* xk = xpass + d * CHUNK_K;
             if (two) {
-                chunk_math(w0, sc0, xk);
-                chunk_math(w1, sc1, xk + CHUNK_K);
+                chunk_math(w0, sc0, x00, x01);
+                chunk_math(w1, sc1, x10, x11);
             } else {
-                chunk_math(w0, sc0, xk);
+                chunk_math(w0, sc0, x00, x01);
             }
         }
         xpass += kGemvRing * CHUNK_K;
