@@ -34,6 +34,15 @@ L2_BYTES_FALLBACK = 126 * 1024 * 1024
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu
+# capture each; figures and commands in profiles/decode_gemv_int4_llama_gate_full.md and
+# profiles/prefill_gemm_pair_int4_llama_ffn_full.md), averaged over the launches bench.py times.
+NCU_TRAFFIC_BYTES = {
+    ("llama31_8b_decode", 1): (33.068e6 + 33.068e6 + 33.089e6) / 3,          # gate, up, down
+    ("llama31_8b_prefill", 2048): (73.6e6 + 73.6e6 + 95.9e6) / 3,            # gate, up, down (reads + y write-back)
+}
+
+
 def load_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -352,7 +361,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama31_8b_decode")
     ap.add_argument("--M", type=int, default=0, help="tokens (default: the workload's first M)")
-    ap.add_argument("--copies", type=int, default=0, help="weight copies rotated (default: enough for 3x L2, >= 4)")
+    ap.add_argument("--copies", type=int, default=0, help="weight copies rotated (default: decode 3x L2 and >= 4, prefill 1.5x L2)")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA-graph replay")
     ap.add_argument("--no-branches", action="store_true",
                     help="decode graph: launch the seven layers strictly one after another (default: q/k/v and "
@@ -389,7 +398,7 @@ def main():
     if stage == "decode":
         copies = args.copies or max(4, -(-3 * l2 // layer_bytes))
     else:
-        copies = args.copies or 1
+        copies = args.copies or max(1, -(-3 * l2 // (2 * layer_bytes)))
     ls = LayerSet(workload, M, copies, device, distinct_copies=True)
     use_graph = (stage == "decode") and not args.no_graph
 
@@ -436,7 +445,8 @@ def main():
         dom_bytes = sum(workload.layers[i].weight_bytes for i in dom_ids) / len(dom_ids)
         achieved = dom_bytes / 1e9 / (dom_ms / 1e3)
         roof = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((workload.name, M)),
+                "peak_source": peaks["source"],
                 "bytes_per_launch": dom_bytes, "us_per_launch": dom_ms * 1e3,
                 "frac_of_nominal_8tbs": achieved / 8000.0}
     else:
@@ -445,8 +455,9 @@ def main():
         dom_flops = sum(workload.layers[i].flops(M) for i in dom_ids) / len(dom_ids)
         achieved = dom_flops / 1e12 / (dom_ms / 1e3)
         peak = peaks["bf16_tflops"]
-        roof = {"bound": "tensor", "kernel": "gemm_kernel<int4, grouped>", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"],
+        roof = {"bound": "tensor", "kernel": "gemm_pair_kernel<int4, grouped>", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": NCU_TRAFFIC_BYTES.get((workload.name, M)),
+                "peak_source": peaks["source"],
                 "flops_per_launch": dom_flops, "us_per_launch": dom_ms * 1e3,
                 "frac_of_nominal_2250": achieved / 2250.0}
 
@@ -488,7 +499,7 @@ def prefill_sub(torch, device, peaks, steps, local):
     w = C.by_name("llama31_8b_prefill")
     M = w.Ms[0]
     try:
-        ls = LayerSet(w, M, 1, device)
+        ls = LayerSet(w, M, 2, device)
         res = bench_stage(torch, ls, "prefill", steps, 3, False, physical_gpu_index(local))
     except P.QLinearError as e:
         return {"unavailable": str(e)}
@@ -500,9 +511,10 @@ def prefill_sub(torch, device, peaks, steps, local):
     return {"metric": "prefill_tflops", "value": tf, "unit": "TFLOP/s", "steps": res["steps"],
             "ms_per_step": res["ms"] / res["steps"], "config": {"workload": w.name, "M": M},
             "clocks": res["clocks"], "gpu_launches": res["launches"],
-            "roofline": {"bound": "tensor", "kernel": "gemm_kernel<int4, grouped>", "achieved": ach,
+            "roofline": {"bound": "tensor", "kernel": "gemm_pair_kernel<int4, grouped>", "achieved": ach,
                          "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
-                         "traffic": None, "peak_source": peaks["source"], "frac_of_nominal_2250": ach / 2250.0}}
+                         "traffic": NCU_TRAFFIC_BYTES.get((w.name, M)), "peak_source": peaks["source"],
+                         "frac_of_nominal_2250": ach / 2250.0}}
 
 
 if __name__ == "__main__":
