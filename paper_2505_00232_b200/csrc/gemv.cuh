@@ -60,6 +60,14 @@ __device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], 
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// D = A.B with a zero accumulator input (no register has to be cleared first).
+__device__ __forceinline__ void mma_16816_zero(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+
 template <int BITS, bool GROUPED, bool XDIRECT>
 __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
 {
@@ -114,9 +122,9 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     // Weights do not depend on the previous kernel: fill the ring before waiting for it.
     if (GROUPED) { copy16(sbuf_u32, ssrc, kc0 + (lane >> 2) < kc1); ssrc += pass_bytes; }
 #pragma unroll
-    for (int d = 0; d < kGemvRing; ++d) {
+    for (int d = 0; d < kGemvRing; ++d) {                                // one commit group per pair of chunks
         copy16(ring_u32 + d * 512, wsrc, kc0 + d < kc1);
-        commit();
+        if (d & 1) commit();
         wsrc += p.block_bytes;
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -142,11 +150,12 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     // independent and those columns are never stored.
     const __half* xpass = XDIRECT ? p.x + (int64_t)min(g, p.M - 1) * p.K + 8 * c + kc0 * CHUNK_K
                                   : xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
-    const __half* xend = p.x + (int64_t)(min(g, p.M - 1) + 1) * p.K;     // direct form: end of this token's row
+    // Direct form: the host chooses it only when K is a whole number of chunks, so every chunk in
+    // [kc0, kc1) lies inside the token's row and the loads need no bounds check.
     auto load_x = [&](const __half* ptr) {
-        uint4 v = make_uint4(0, 0, 0, 0);
+        uint4 v;
         if (!XDIRECT) v = *reinterpret_cast<const uint4*>(ptr);
-        else if (ptr < xend) asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
+        else asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
         return v;
     };
     const unsigned char* wslot = ring + lane * 16;
@@ -161,9 +170,9 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             for (int h = 0; h < 2; ++h) {
                 const uint4 xv = h == 0 ? xa : xb;
                 if (GROUPED) {
-                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    float acc[4];
                     unpack_int4_word(ww[2 * h], a);
-                    mma_16816_pure(acc, a, xv.x, xv.y);
+                    mma_16816_zero(acc, a, xv.x, xv.y);
                     unpack_int4_word(ww[2 * h + 1], a);
                     mma_16816_pure(acc, a, xv.z, xv.w);
                     const __half2 s_lo = *reinterpret_cast<const __half2*>(&sc.x);          // row g:   G0, G1
@@ -199,10 +208,11 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             const bool two = kc + d + 1 < kc1;
             // x fragments first: their latency (L1 / shared) runs under the wait for the weights
             const __half* xk = xpass + d * CHUNK_K;
-            const uint4 x00 = load_x(xk), x10 = load_x(xk + CHUNK_K);
+            const __half* xk1 = two ? xk + CHUNK_K : xk;                 // odd tail: stay inside the row
+            const uint4 x00 = load_x(xk), x10 = load_x(xk1);
             uint4 x01 = x00, x11 = x10;
-            if (BITS == 4) { x01 = load_x(xk + 32); x11 = load_x(xk + CHUNK_K + 32); }
-            asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing - 2) : "memory");
+            if (BITS == 4) { x01 = load_x(xk + 32); x11 = load_x(xk1 + 32); }
+            asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing / 2 - 1) : "memory");
             if (GROUPED && d == 0) {
                 __syncwarp();                                            // scales of this pass visible; last pass's reads done
                 copy16(sbuf_u32 + (sflip ^ 1) * 512, ssrc, kc + kGemvRing + (lane >> 2) < kc1);
@@ -215,8 +225,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
                 sc0 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + d * 64 + g * 8);
                 sc1 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + (d + 1) * 64 + g * 8);
             }
-            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slots just read
-            commit();
+            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slots just read (one group)
             copy16(ring_u32 + (d + 1) * 512, wsrc + p.block_bytes, kc + d + 1 + kGemvRing < kc1);
             commit();
             wsrc += 2 * (int64_t)p.block_bytes;

@@ -73,7 +73,10 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             if ((ks - 1) * cps >= L.n_kc && ks > 1) continue;               // would leave a slice empty
             const int span = std::min(ks_cta * cps, L.n_kc) * L.chunk_k;
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
-            const int x_bytes = env_int("QLINEAR_GEMV_XDIRECT", 1) ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
+            // x fragments straight from global memory need K to be a whole number of chunks (no bounds checks
+            // in the kernel); otherwise x is staged in shared memory with zeros beyond K
+            const bool direct = env_int("QLINEAR_GEMV_XDIRECT", 1) && (L.K % L.chunk_k) == 0;
+            const int x_bytes = direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
