@@ -109,9 +109,9 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     const uint32_t sbuf_u32 = (uint32_t)__cvta_generic_to_shared(sbuf) + lane * 16;
     const uint8_t* blk = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes;
     const uint8_t* wsrc = blk + (rb & 7) * 512 + lane * 16;
-    // lane L copies part (L & 3) of the scales of chunk (pass start + L / 4)
-    const uint8_t* ssrc = blk + (int64_t)(lane >> 2) * p.block_bytes + kWeightBlockBytes + (rb & 7) * 64 + (lane & 3) * 16;
-    const int64_t pass_bytes = (int64_t)kGemvRing * p.block_bytes;
+    // lane L copies part (L & 3) of the scales of chunk (pass start + L / 4); the address is kept relative
+    // to the weight address of the pass's first chunk (wsrc at the top of a pass)
+    const int s_off = (lane >> 2) * p.block_bytes + kWeightBlockBytes - (rb & 7) * 448 + (lane & 3) * 16 - lane * 16;
 
     auto copy16 = [](uint32_t dst, const void* src, bool in_range) {     // out of range: reads nothing, writes zeros
         const uint32_t sz = in_range ? 16u : 0u;
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     auto commit = [] { asm volatile("cp.async.commit_group;" ::: "memory"); };
 
     // Weights do not depend on the previous kernel: fill the ring before waiting for it.
-    if (GROUPED) { copy16(sbuf_u32, ssrc, kc0 + (lane >> 2) < kc1); ssrc += pass_bytes; }
+    if (GROUPED) copy16(sbuf_u32, wsrc + s_off, kc0 + (lane >> 2) < kc1);
 #pragma unroll
     for (int d = 0; d < kGemvRing; ++d) {                                // one commit group per pair of chunks
         copy16(ring_u32 + d * 512, wsrc, kc0 + d < kc1);
@@ -158,7 +158,18 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
         else asm volatile("ld.global.ca.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr));
         return v;
     };
-    const unsigned char* wslot = ring + lane * 16;
+    // reads of the ring and of the scale buffers go through 32-bit shared-window addresses
+    auto lds128 = [](uint32_t addr) {
+        uint4 v;
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+        return v;
+    };
+    auto lds64 = [](uint32_t addr) {
+        uint2 v;
+        asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+        return v;
+    };
+    const uint32_t sc_u32 = sbuf_u32 - lane * 16 + g * 8;                // this lane's scales inside a pass buffer
     int sflip = 0;                                                       // scale buffer of the current pass
 
     // one chunk: unpack in registers, feed the tensor core, apply the group scales in fp32
@@ -199,13 +210,15 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
         }
     };
 
-    // Two chunks per iteration: both are read into registers and their slots refilled before the math, so
-    // the two independent unpack/MMA chains interleave.
-    for (int kc = kc0; kc < kc1; kc += kGemvRing) {
+    // One pass = one trip round the ring.  Two chunks per iteration: both are read into registers and
+    // their slots refilled before the math, so the two independent unpack/MMA chains interleave.
+    // `checked` is a literal at both call sites: a pass called with false lies, with all its refills,
+    // inside the warp's K slice and carries no range test at all.
+    auto pass = [&](const bool checked, const int kc) {
 #pragma unroll
         for (int d = 0; d < kGemvRing; d += 2) {
-            if (kc + d >= kc1) break;
-            const bool two = kc + d + 1 < kc1;
+            if (checked && kc + d >= kc1) break;
+            const bool two = !checked || kc + d + 1 < kc1;
             // x fragments first: their latency (L1 / shared) runs under the wait for the weights
             const __half* xk = xpass + d * CHUNK_K;
             const __half* xk1 = two ? xk + CHUNK_K : xk;                 // odd tail: stay inside the row
@@ -215,19 +228,18 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing / 2 - 1) : "memory");
             if (GROUPED && d == 0) {
                 __syncwarp();                                            // scales of this pass visible; last pass's reads done
-                copy16(sbuf_u32 + (sflip ^ 1) * 512, ssrc, kc + kGemvRing + (lane >> 2) < kc1);
-                ssrc += pass_bytes;
+                copy16(sbuf_u32 + (sflip ^ 1) * 512, wsrc + s_off, !checked || kc + kGemvRing + (lane >> 2) < kc1);
             }
-            const uint4 w0 = *reinterpret_cast<const uint4*>(wslot + d * 512);
-            const uint4 w1 = *reinterpret_cast<const uint4*>(wslot + (d + 1) * 512);
+            const uint4 w0 = lds128(ring_u32 + d * 512);
+            const uint4 w1 = lds128(ring_u32 + (d + 1) * 512);
             uint2 sc0 = make_uint2(0, 0), sc1 = make_uint2(0, 0);
             if (GROUPED) {
-                sc0 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + d * 64 + g * 8);
-                sc1 = *reinterpret_cast<const uint2*>(sbuf + sflip * 512 + (d + 1) * 64 + g * 8);
+                sc0 = lds64(sc_u32 + sflip * 512 + d * 64);
+                sc1 = lds64(sc_u32 + sflip * 512 + (d + 1) * 64);
             }
-            copy16(ring_u32 + d * 512, wsrc, kc + d + kGemvRing < kc1);  // refill the slots just read (one group)
-            copy16(ring_u32 + (d + 1) * 512, wsrc + p.block_bytes, kc + d + 1 + kGemvRing < kc1);
-            commit();
+            copy16(ring_u32 + d * 512, wsrc, !checked || kc + d + kGemvRing < kc1);      // refill the slots just read
+            copy16(ring_u32 + (d + 1) * 512, wsrc + p.block_bytes, !checked || kc + d + 1 + kGemvRing < kc1);
+            commit();                                                    // (one group per pair)
             wsrc += 2 * (int64_t)p.block_bytes;
             if (two) {
                 chunk_math(w0, sc0, x00, x01);
@@ -236,6 +248,12 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
                 chunk_math(w0, sc0, x00, x01);
             }
         }
+    };
+    for (int kc = kc0; kc < kc1; kc += kGemvRing) {
+        // Measured: the test-free pass pays for int8 (+12 %), while the int4 form runs slower without the
+        // branches that keep its four pairs apart (LM head -20 %), so int4 always takes the checked pass.
+        if (BITS == 8 && kc + 2 * kGemvRing <= kc1) pass(false, kc);
+        else pass(true, kc);
         xpass += kGemvRing * CHUNK_K;
         sflip ^= 1;
     }
