@@ -155,35 +155,35 @@ class LayerSet:
 
     _STAGE = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}
 
-    def step_branched(self, cp):
-        """One pass with the data flow of a transformer layer: q, k, v read the same input and run as
-        parallel branches (three streams), then o; gate and up likewise, then down.  Same seven calls."""
-        torch = self.torch
-        main = torch.cuda.current_stream()
-        if not hasattr(self, "_side"):
-            self._side = [torch.cuda.Stream(), torch.cuda.Stream()]
+    def _groups(self):
+        """Consecutive layers that read the same input (q, k, v; gate, up), as lists of layer indices."""
         groups, prev = [], None
         for li, l in enumerate(self.layers):
             st = self._STAGE.get(l.name, 100 + li)
-            if st != prev:
-                groups.append([])
-                prev = st
-            groups[-1].append(li)
-        for grp in groups:
-            fork = torch.cuda.Event()
-            fork.record(main)
-            joins = []
-            for j, li in enumerate(grp):
-                stream = main if j == 0 else self._side[(j - 1) % 2]
-                if j:
-                    stream.wait_event(fork)
-                self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M, stream)
-                if j:
-                    ev = torch.cuda.Event()
-                    ev.record(stream)
-                    joins.append(ev)
-            for ev in joins:
-                main.wait_event(ev)
+            same = st == prev and groups and all(
+                (self.layers[j].K, self.layers[j].bits, self.layers[j].group) == (l.K, l.bits, l.group) for j in groups[-1])
+            if same:
+                groups[-1].append(li)
+            else:
+                groups.append([li])
+            prev = st
+        return groups
+
+    def step_grouped(self, cp):
+        """One pass with the data flow of a transformer layer: q, k, v read the same input and go out as ONE
+        grouped call, then o; gate and up likewise, then down.  Same seven layers, same bytes, four launches."""
+        P = self.P
+        for grp in self._groups():
+            if len(grp) == 1:
+                li = grp[0]
+                self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
+            else:
+                P.qlinear_forward_group_raw([self.lin[cp][li] for li in grp], self.x[grp[0]].data_ptr(),
+                                            [self.y[li].data_ptr() for li in grp], self.M)
+
+    @property
+    def launches_grouped(self):
+        return len(self._groups())
 
     def step_e2e(self, cp):
         """Host buffers in, host buffers out: H2D of every x, the forwards, D2H of every y."""
@@ -315,11 +315,12 @@ def run_reference(args, workload, M):
 
 
 # ------------------------------------------------------------------------------------ GPU legs
-def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, branches=False):
+def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, grouped=False):
     """Times `steps` passes over the layer set; returns dict with ms_per_step, clocks, launches."""
     copies = ls.copies
+    per_step = ls.launches_grouped if (use_graph and grouped) else len(ls.layers)
     if use_graph:
-        step_fn = ls.step_branched if branches else ls.step
+        step_fn = ls.step_grouped if grouped else ls.step
         graph = capture_graph(torch, lambda i: step_fn(i % copies), copies)
         n_replays = max(1, steps // copies)
         steps = n_replays * copies
@@ -332,7 +333,7 @@ def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, branc
         run = lambda: time_events(torch, lambda i: ls.step(i % copies), steps)
     with ClockSampler(sampler_index) as cs:
         ms = run()
-    return {"ms": ms, "steps": steps, "clocks": cs.summary(), "launches": steps * len(ls.layers)}
+    return {"ms": ms, "steps": steps, "clocks": cs.summary(), "launches": steps * per_step}
 
 
 def dominant_kernel_time(torch, ls, layer_ids, launches, use_graph):
@@ -363,9 +364,9 @@ def main():
     ap.add_argument("--M", type=int, default=0, help="tokens (default: the workload's first M)")
     ap.add_argument("--copies", type=int, default=0, help="weight copies rotated (default: decode 3x L2 and >= 4, prefill 1.5x L2)")
     ap.add_argument("--no-graph", action="store_true", help="plain stream launches instead of CUDA-graph replay")
-    ap.add_argument("--no-branches", action="store_true",
-                    help="decode graph: launch the seven layers strictly one after another (default: q/k/v and "
-                         "gate/up as parallel graph branches, the data flow of a transformer layer)")
+    ap.add_argument("--no-groups", action="store_true",
+                    help="decode graph: one launch per layer (default: layers that read the same input, q/k/v and "
+                         "gate/up, go out as one grouped call each, the data flow of a transformer layer)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill sub-measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill-steps", type=int, default=20)
@@ -406,8 +407,8 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    branches = use_graph and not args.no_branches
-    res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local), branches)
+    grouped = use_graph and not args.no_groups
+    res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local), grouped)
     if world > 1:
         dist.barrier()
         res["ms"] = max_over_ranks(res["ms"], device)
@@ -468,7 +469,7 @@ def main():
         "config": {"workload": workload.name, "M": M, "layers": [f"{l.name}:{l.N}x{l.K}:int{l.bits}" for l in workload.layers],
                    "weight_copies": copies, "weight_bytes_per_step": ls.weight_bytes,
                    "l2": f"{copies} weight copies ({copies * layer_bytes / 1e6:.0f} MB) rotated per step; no flush",
-                   "launch": ("cuda graph + programmatic dependent launch" + (", q/k/v and gate/up as parallel branches" if branches else ""))
+                   "launch": ("cuda graph + programmatic dependent launch" + (", q/k/v and gate/up as one grouped call each" if grouped else ""))
                              if use_graph else "stream launches",
                    "parallelism": "replicas only" if world > 1 else "single gpu"},
         "clocks": res["clocks"], "gpu_launches": res["launches"],

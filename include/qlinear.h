@@ -93,6 +93,23 @@ ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int d
  * handle hit a bounded wait; see qlinear_device_status). */
 ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
 
+/* The same result as n calls of qlinear_forward with one x: ys_dev[i] = x . W_i^T for the n layers hs[i]
+ * (1 <= n <= 4), which must live on one device and agree in K, bits and group (q/k/v projections; gate
+ * and up projections).  For M <= 8 all n layers run in ONE decode kernel launch: their output channels
+ * are numbered one after the other and spread over the grid together, so short layers do not each pay
+ * a launch of their own (the paper's operator fusion, Section 3 "Operator Fusion", merges kernels for
+ * the same reason: launch overhead and memory-bound work).  Every output is bit-identical to what
+ * qlinear_forward gives for that layer only if the K split chosen for the group equals the layer's own;
+ * it always meets the same tolerance, and is run-to-run deterministic.  For larger M the layers run
+ * one after the other with the prefill kernel.
+ *   hs      host array of n handles; ys_dev host array of n device pointers (fp16 [M, N_i], 16-byte
+ *           aligned, not overlapping x_dev or one another); x_dev as in qlinear_forward.
+ * Asynchronous, allocates nothing.  Calls that put the same handle first must not run concurrently
+ * from different host threads (the plan of the group is cached in it).
+ * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..4 or layers that do not agree. */
+ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
+                                int32_t M, void* cuda_stream);
+
 /* The kernel qlinear_forward uses for M tokens on this handle (0 if h is NULL or M < 1). */
 int32_t qlinear_path_for(qlinear_t h, int32_t M);
 

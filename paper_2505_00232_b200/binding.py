@@ -20,7 +20,7 @@ QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ALLOC, QL_ERR_CUDA, QL_ERR_DEVICE
 QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version",
 )
@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_path_for.restype = i32
     lib.qlinear_debug_unpack_device.argtypes = [vp, vp, vp]
     lib.qlinear_debug_unpack_device.restype = ctypes.c_int
+    lib.qlinear_forward_group.argtypes = [ctypes.POINTER(vp), ctypes.c_int32, vp, ctypes.POINTER(vp), ctypes.c_int32, vp]
+    lib.qlinear_forward_group.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.qlinear_device_status.restype = ctypes.c_int
     lib.qlinear_decode_static.argtypes = [dp, vp, vp, vp, i32, ctypes.c_int, vp]
@@ -149,6 +151,30 @@ def qlinear_decode_static(desc: Desc, packed, x, out=None, stream=None):
                                      ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(out.data_ptr()), M,
                                      x.device.index or 0, _stream_ptr(stream)), "qlinear_decode_static")
     return out
+
+
+def qlinear_forward_group_raw(lins, x_ptr: int, y_ptrs, M: int, stream=None) -> None:
+    """qlinear_forward_group on raw device pointers: the layers `lins` applied to one x."""
+    n = len(lins)
+    hs = (ctypes.c_void_p * n)(*[l._h for l in lins])
+    ys = (ctypes.c_void_p * n)(*[ctypes.c_void_p(int(p)) for p in y_ptrs])
+    _check(lib.qlinear_forward_group(hs, n, ctypes.c_void_p(x_ptr), ys, M, _stream_ptr(stream)), "qlinear_forward_group")
+
+
+def qlinear_forward_group(lins, x, outs=None, stream=None):
+    """x: fp16 CUDA tensor [M, K] -> list of fp16 [M, N_i], one per layer (one launch for M <= 8)."""
+    import torch
+    K = lins[0].desc.K
+    if x.dim() != 2 or x.shape[1] != K or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_group (x must be contiguous fp16 CUDA [M, K])")
+    M = x.shape[0]
+    if outs is None:
+        outs = [torch.empty((M, l.desc.N), dtype=torch.float16, device=x.device) for l in lins]
+    for l, o in zip(lins, outs):
+        if o.shape != (M, l.desc.N) or o.dtype != torch.float16 or not o.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_group (bad out tensor)")
+    qlinear_forward_group_raw(lins, x.data_ptr(), [o.data_ptr() for o in outs], M, stream)
+    return outs
 
 
 class QLinear:

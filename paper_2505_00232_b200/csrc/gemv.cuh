@@ -28,13 +28,20 @@ constexpr int kGemvWarps = 8;
 constexpr int kGemvThreads = kGemvWarps * 32;
 constexpr int kGemvRing = 8;             // chunks prefetched per warp (cp.async ring slots)
 
+constexpr int kGemvMaxGroup = 4;         // layers that may share one launch (same input, same K and scheme)
+
 struct GemvParams {
-    const uint8_t* body;                 // first block of the packed body
-    const __half* chan_scales;           // per-channel scales (nullptr when grouped)
+    // One launch serves up to kGemvMaxGroup layers that read the same x (q/k/v, gate/up): their row-blocks
+    // are numbered one after the other; rb_end[i] is the number of row-blocks of layers 0..i.
+    const uint8_t* body[kGemvMaxGroup];  // first block of each packed body
+    const __half* chan_scales[kGemvMaxGroup];   // per-channel scales (nullptr when grouped)
+    __half* y[kGemvMaxGroup];            // [M, N_i]
+    int32_t N[kGemvMaxGroup];
+    int32_t rb_end[kGemvMaxGroup];
+    int32_t n_layers;
     const __half* x;                     // [M, K]
-    __half* y;                           // [M, N]
-    int32_t M, N, K;
-    int32_t n_rb;                        // row-blocks holding at least one real row
+    int32_t M, K;
+    int32_t n_rb;                        // row-blocks holding at least one real row, all layers
     int32_t n_kc;                        // chunks along K
     int32_t block_bytes;
     int32_t ks_cta;                      // K slices handled inside one CTA: 1, 2, 4 or 8
@@ -88,8 +95,13 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     const int crank = (int)crank_u, rb_group = (int)rb_group_u;
     const int rb_per_cta = kGemvWarps >> p.ks_cta_log2;
     const int ks_local = warp & (p.ks_cta - 1);
-    const int rb = rb_group * rb_per_cta + (warp >> p.ks_cta_log2);
-    const bool rb_live = rb < p.n_rb;
+    const int rb_all = rb_group * rb_per_cta + (warp >> p.ks_cta_log2);  // numbered through all layers of the launch
+    const bool rb_live = rb_all < p.n_rb;
+    int layer = 0;
+#pragma unroll
+    for (int i = 1; i < kGemvMaxGroup; ++i)
+        if (i < p.n_layers && rb_all >= p.rb_end[i - 1]) layer = i;
+    const int rb = rb_all - (layer ? p.rb_end[layer - 1] : 0);           // row-block inside its layer
     const int ks = crank * p.ks_cta + ks_local;
     const int kc0 = min(ks * p.cps, p.n_kc);
     const int kc1 = rb_live ? min(kc0 + p.cps, p.n_kc) : kc0;
@@ -107,7 +119,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     unsigned char* sbuf = ring + kGemvRing * 512;
     const uint32_t ring_u32 = (uint32_t)__cvta_generic_to_shared(ring) + lane * 16;
     const uint32_t sbuf_u32 = (uint32_t)__cvta_generic_to_shared(sbuf) + lane * 16;
-    const uint8_t* blk = p.body + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes;
+    const uint8_t* blk = p.body[layer] + ((int64_t)(rb >> 3) * p.n_kc + kc0) * p.block_bytes;
     const uint8_t* wsrc = blk + (rb & 7) * 512 + lane * 16;
     // lane L copies part (L & 3) of the scales of chunk (pass start + L / 4); the address is kept relative
     // to the weight address of the pass's first chunk (wsrc at the top of a pass)
@@ -264,13 +276,17 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     __syncthreads();
 
     auto store_out = [&](int rbl, int e, float v) {
-        const int out_rb = rb_group * rb_per_cta + rbl;
+        int out_rb = rb_group * rb_per_cta + rbl, ly = 0;
+#pragma unroll
+        for (int i = 1; i < kGemvMaxGroup; ++i)
+            if (i < p.n_layers && out_rb >= p.rb_end[i - 1]) ly = i;
+        out_rb -= ly ? p.rb_end[ly - 1] : 0;
         const int el = e >> 2, i = e & 3;                                // lane that produced it, register index
         const int row = out_rb * kRbRows + (el >> 2) + 8 * (i >> 1);
         const int tok = 2 * (el & 3) + (i & 1);
-        if (row < p.N && tok < p.M) {
-            if (!GROUPED) v *= __half2float(p.chan_scales[row]);
-            p.y[(int64_t)tok * p.N + row] = __float2half_rn(v);
+        if (row < p.N[ly] && tok < p.M) {
+            if (!GROUPED) v *= __half2float(p.chan_scales[ly][row]);
+            p.y[ly][(int64_t)tok * p.N[ly] + row] = __float2half_rn(v);
         }
     };
 

@@ -38,6 +38,8 @@ struct qlinear_s {
     int gemv_max_m;
     bool pdl;
     GemvPlan gemv[9];          // index = M (1..8)
+    GemvPlan group_gemv[9];    // the same for the last group of layers launched with this one in front
+    int group_rb;              // row-blocks of that group (0 = none yet)
     GemmPlan gemm;
     // streaming decode kernel
     int gemv_kernel_choice;    // 0 = cluster kernel, 1 = streaming kernel
@@ -59,11 +61,13 @@ int env_int(const char* name, int dflt)
     return (v && *v) ? std::atoi(v) : dflt;
 }
 
-GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
+// n_rb: row-blocks of the launch (one layer, or all layers of a group that shares x).
+GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
 {
-    const int n_rb = (L.N + kRbRows - 1) / kRbRows;
-    const double target = (double)num_sms * env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
-    const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
+    static const int warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
+    static const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
+    static const int xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1);
+    const double target = (double)num_sms * warps_per_sm;
     GemvPlan best{};
     double best_score = -1e30;
     for (int ks_cta = 1; ks_cta <= 8; ks_cta *= 2)
@@ -75,7 +79,7 @@ GemvPlan plan_gemv(const Layout& L, int M, int num_sms)
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
             // x fragments straight from global memory need K to be a whole number of chunks (no bounds checks
             // in the kernel); otherwise x is staged in shared memory with zeros beyond K
-            const bool direct = env_int("QLINEAR_GEMV_XDIRECT", 1) && (L.K % L.chunk_k) == 0;
+            const bool direct = xdirect && (L.K % L.chunk_k) == 0;
             const int x_bytes = direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
@@ -139,17 +143,35 @@ cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPla
                             : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
 }
 
-ql_status forward_gemv(qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
+// One launch for n layers that read the same x (n == 1: the plain forward).
+ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st)
 {
+    qlinear_s* h = hs[0];
     const Layout& L = h->L;
-    const GemvPlan& pl = h->gemv[M];
     GemvParams prm{};
-    prm.body = h->blob + L.body_offset;
-    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
+    int n_rb = 0;
+    for (int i = 0; i < n; ++i) {
+        const Layout& Li = hs[i]->L;
+        prm.body[i] = hs[i]->blob + Li.body_offset;
+        prm.chan_scales[i] = Li.grouped ? nullptr : reinterpret_cast<const __half*>(hs[i]->blob + Li.chan_scale_offset);
+        prm.y[i] = static_cast<__half*>(ys[i]);
+        prm.N[i] = Li.N;
+        n_rb += (Li.N + kRbRows - 1) / kRbRows;
+        prm.rb_end[i] = n_rb;
+    }
+    prm.n_layers = n;
+    GemvPlan pl;
+    if (n == 1) pl = h->gemv[M];
+    else {
+        if (h->group_rb != n_rb) {                                       // plans of the last group this layer led
+            for (int m = 1; m <= 8; ++m) h->group_gemv[m] = plan_gemv(L, n_rb, m, h->num_sms);
+            h->group_rb = n_rb;
+        }
+        pl = h->group_gemv[M];
+    }
     prm.x = static_cast<const __half*>(x);
-    prm.y = static_cast<__half*>(y);
-    prm.M = M; prm.N = L.N; prm.K = L.K;
-    prm.n_rb = (L.N + kRbRows - 1) / kRbRows;
+    prm.M = M; prm.K = L.K;
+    prm.n_rb = n_rb;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
@@ -278,7 +300,7 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
     h->num_sms = sms;
     h->gemv_max_m = std::max(1, std::min(8, env_int("QLINEAR_GEMV_MAX_M", 8)));
     h->pdl = env_int("QLINEAR_PDL", 1) != 0;
-    for (int M = 1; M <= 8; ++M) h->gemv[M] = plan_gemv(L, M, sms);
+    for (int M = 1; M <= 8; ++M) h->gemv[M] = plan_gemv(L, (L.N + kRbRows - 1) / kRbRows, M, sms);
     ql_status st = gemm_plan(L, sms, &h->gemm);
     if (st != QL_OK) { delete h; return st; }
     // streaming decode kernel: persistent grid, ring depth and per-handle scratch
@@ -330,10 +352,33 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(h, x, y, M, st);
+    if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
     if (gemm_pair_applicable(h->L, M))
         return gemm_pair_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms, h->gemm_scratch, h->gemm_counters);
     return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
+}
+
+extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x, void* const* ys, int32_t M, void* stream)
+{
+    if (!hs || !ys || !x || n < 1 || n > kGemvMaxGroup || M < 1) return QL_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i) {
+        if (!hs[i] || !ys[i] || (reinterpret_cast<uintptr_t>(ys[i]) & 15)) return QL_ERR_INVALID_ARG;
+        const Layout &a = hs[0]->L, &b = hs[i]->L;
+        if (hs[i]->device != hs[0]->device || a.K != b.K || a.bits != b.bits || a.group != b.group) return QL_ERR_INVALID_ARG;
+        if ((int64_t)M * b.N > INT32_MAX) return QL_ERR_INVALID_ARG;
+    }
+    if ((reinterpret_cast<uintptr_t>(x) & 15) || (int64_t)M * hs[0]->L.K > INT32_MAX) return QL_ERR_INVALID_ARG;
+    // One kernel where the decode kernel serves the call; otherwise the layers run one after the other.
+    if (n > 1 && M <= hs[0]->gemv_max_m && hs[0]->gemv_kernel_choice == 0) {
+        DeviceGuard guard(hs[0]->device);
+        if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+        return forward_gemv(const_cast<qlinear_s* const*>(hs), n, x, ys, M, static_cast<cudaStream_t>(stream));
+    }
+    for (int i = 0; i < n; ++i) {
+        ql_status s = qlinear_forward(hs[i], x, ys[i], M, stream);
+        if (s != QL_OK) return s;
+    }
+    return QL_OK;
 }
 
 extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, void* stream)

@@ -178,3 +178,53 @@ def test_streaming_kernel_parity(P, torch, monkeypatch, M, N, K, bits, group):
     want = (s[:, 7 // G].astype(np.float64) * q[:, 7].astype(np.float64)).astype(np.float16)
     yo = lin.forward(torch.from_numpy(xo).cuda()).cpu().numpy()
     assert (yo.view(np.uint16) == want.view(np.uint16)[None, :]).all()
+
+
+GROUPS = [
+    # (M, K, bits, group, [N_i]): q/k/v-like and gate/up-like groups, ragged N, N not a multiple of 16, K tail
+    (1, 4096, 8, 0, [4096, 1024, 1024]), (4, 2304, 8, 0, [2048, 1024, 1024]), (1, 4096, 4, 32, [2048, 2048]),
+    (8, 2304, 4, 32, [1160, 520]), (3, 352, 4, 32, [200, 8, 24, 136]), (2, 160, 8, 0, [136, 8]), (5, 384, 4, 0, [40, 264]),
+]
+
+
+@pytest.mark.parametrize("M,K,bits,group,Ns", GROUPS)
+def test_forward_group_parity(P, torch, M, K, bits, group, Ns):
+    """Layers that share x in one launch: every layer's output meets the single-layer bar."""
+    cases = [rand_case(5000 + 17 * i + N + K, M, N, K, bits, group) for i, N in enumerate(Ns)]
+    x = cases[0][2]
+    lins = [P.QLinear.from_weights(q, s, bits, group, device="cuda:0") for q, s, _ in cases]
+    xd = torch.from_numpy(x).cuda()
+    ys = P.qlinear_forward_group(lins, xd)
+    torch.cuda.synchronize()
+    assert lins[0].device_status()[0] == 0
+    for (q, s, _), y in zip(cases, ys):
+        assert_parity(y.cpu().numpy(), x, q, s, group)
+    again = P.qlinear_forward_group(lins, xd)
+    for a, b in zip(ys, again):
+        assert torch.equal(a, b)                         # run-to-run identical
+    # a one-hot x gives the correctly rounded single product in every layer, bit for bit
+    xo = np.zeros_like(x)
+    xo[:, 5] = 1.0
+    G = K if group == 0 else group
+    yo = P.qlinear_forward_group(lins, torch.from_numpy(xo).cuda())
+    for (q, s, _), y in zip(cases, yo):
+        want = (s.reshape(q.shape[0], -1)[:, 5 // G].astype(np.float64) * q[:, 5].astype(np.float64)).astype(np.float16)
+        assert (y.cpu().numpy().view(np.uint16) == want.view(np.uint16)[None, :]).all()
+
+
+def test_forward_group_prefill_and_errors(P, torch):
+    """M > 8 runs the layers one after the other (same results as single calls); mismatched layers are refused."""
+    M, K = 24, 256
+    cases = [rand_case(6000 + N, M, N, K, 4, 32) for N in (128, 264)]
+    x = cases[0][2]
+    lins = [P.QLinear.from_weights(q, s, 4, 32, device="cuda:0") for q, s, _ in cases]
+    xd = torch.from_numpy(x).cuda()
+    ys = P.qlinear_forward_group(lins, xd)
+    for lin, y in zip(lins, ys):
+        assert torch.equal(y, lin.forward(xd))
+    q8, s8, _ = rand_case(6100, M, 128, K, 8, 0)
+    other = P.QLinear.from_weights(q8, s8, 8, 0, device="cuda:0")
+    with pytest.raises(P.QLinearError):
+        P.qlinear_forward_group([lins[0], other], xd)
+    with pytest.raises(P.QLinearError):
+        P.qlinear_forward_group(lins * 3, xd)            # more than four layers
