@@ -64,9 +64,9 @@ int env_int(const char* name, int dflt)
 // n_rb: row-blocks of the launch (one layer, or all layers of a group that shares x).
 GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
 {
-    static const int warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
-    static const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
-    static const int xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1);
+    const int warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
+    const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
+    const int xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1);
     const double target = (double)num_sms * warps_per_sm;
     GemvPlan best{};
     double best_score = -1e30;
@@ -85,7 +85,10 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
             const double eff = (double)L.n_kc / ((double)ks * cps);
-            double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 2 ? 1.0 : 0.0);
+            // slices of fewer than 4 chunks never reach a steady state (measured: 2-chunk slices lose to 4-chunk
+            // slices on half as many warps)
+            double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 4 ? 1.25 : 0.0) - (cps < 2 ? 1.0 : 0.0);
+            if (warps > target) score -= 2.0;                               // more CTAs than fit at once: a second wave
             if (force_ks) score = (ks == force_ks) ? 0.0 : -1e29;
             if (score > best_score) {
                 best_score = score;
