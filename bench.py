@@ -35,10 +35,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu
-# capture each; figures and commands in profiles/decode_gemv_int4_llama_gate_full.md and
+# capture each; figures and commands in profiles/decode_gemv_int4_llama_gate_up_full.md and
 # profiles/prefill_gemm_pair_int4_llama_ffn_full.md), averaged over the launches bench.py times.
 NCU_TRAFFIC_BYTES = {
-    ("llama31_8b_decode", 1): (33.068e6 + 33.068e6 + 33.089e6) / 3,          # gate, up, down
+    ("llama31_8b_decode", 1): (66.095104e6 + 0.455936e6 + 33.085440e6) / 2,     # gate+up and down launches
     ("llama31_8b_prefill", 2048): (73.6e6 + 73.6e6 + 95.9e6) / 3,            # gate, up, down (reads + y write-back)
 }
 
@@ -169,11 +169,13 @@ class LayerSet:
             prev = st
         return groups
 
-    def step_grouped(self, cp):
+    def step_grouped(self, cp, only=None):
         """One pass with the data flow of a transformer layer: q, k, v read the same input and go out as ONE
         grouped call, then o; gate and up likewise, then down.  Same seven layers, same bytes, four launches."""
         P = self.P
         for grp in self._groups():
+            if only is not None and not all(li in only for li in grp):
+                continue
             if len(grp) == 1:
                 li = grp[0]
                 self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
@@ -185,17 +187,24 @@ class LayerSet:
     def launches_grouped(self):
         return len(self._groups())
 
-    def step_e2e(self, cp):
-        """Host buffers in, host buffers out: H2D of every x, the forwards, D2H of every y."""
-        for li in range(len(self.layers)):
-            self.x[li].copy_(self.x_host[li], non_blocking=True)
-            self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
-            self.y_host[li].copy_(self.y[li], non_blocking=True)
+    def step_e2e(self, cp, grouped=False):
+        """Host buffers in, host buffers out: H2D of every input, the forwards, D2H of every y."""
+        groups = self._groups() if grouped else [[li] for li in range(len(self.layers))]
+        for grp in groups:
+            li0 = grp[0]
+            self.x[li0].copy_(self.x_host[li0], non_blocking=True)
+            if len(grp) == 1:
+                self.lin[cp][li0].forward_raw(self.x[li0].data_ptr(), self.y[li0].data_ptr(), self.M)
+            else:
+                self.P.qlinear_forward_group_raw([self.lin[cp][li] for li in grp], self.x[li0].data_ptr(),
+                                                 [self.y[li].data_ptr() for li in grp], self.M)
+            for li in grp:
+                self.y_host[li].copy_(self.y[li], non_blocking=True)
         self.torch.cuda.current_stream().synchronize()
 
-    @property
-    def h2d_bytes(self):
-        return sum(2 * self.M * l.K for l in self.layers)
+    def h2d_bytes(self, grouped=False):
+        groups = self._groups() if grouped else [[li] for li in range(len(self.layers))]
+        return sum(2 * self.M * self.layers[g[0]].K for g in groups)
 
     @property
     def d2h_bytes(self):
@@ -318,9 +327,9 @@ def run_reference(args, workload, M):
 def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, grouped=False):
     """Times `steps` passes over the layer set; returns dict with ms_per_step, clocks, launches."""
     copies = ls.copies
-    per_step = ls.launches_grouped if (use_graph and grouped) else len(ls.layers)
+    per_step = ls.launches_grouped if grouped else len(ls.layers)
+    step_fn = ls.step_grouped if grouped else ls.step
     if use_graph:
-        step_fn = ls.step_grouped if grouped else ls.step
         graph = capture_graph(torch, lambda i: step_fn(i % copies), copies)
         n_replays = max(1, steps // copies)
         steps = n_replays * copies
@@ -329,29 +338,33 @@ def bench_stage(torch, ls, stage, steps, warmup, use_graph, sampler_index, group
         run = lambda: time_events(torch, lambda i: graph.replay(), n_replays)
     else:
         for i in range(warmup):
-            ls.step(i % copies)
-        run = lambda: time_events(torch, lambda i: ls.step(i % copies), steps)
+            step_fn(i % copies)
+        run = lambda: time_events(torch, lambda i: step_fn(i % copies), steps)
     with ClockSampler(sampler_index) as cs:
         ms = run()
     return {"ms": ms, "steps": steps, "clocks": cs.summary(), "launches": steps * per_step}
 
 
-def dominant_kernel_time(torch, ls, layer_ids, launches, use_graph):
-    """Average device time per launch of the listed layers' kernel, rotated over the weight copies."""
+def dominant_kernel_time(torch, ls, layer_ids, launches, use_graph, grouped=False):
+    """Average device time per launch of the listed layers' kernel, rotated over the weight copies.
+    Returns (ms per launch, launches per pass): with grouped calls a pass over the listed layers is
+    fewer launches than layers."""
     copies = ls.copies
+    step_fn = (lambda cp: ls.step_grouped(cp, only=layer_ids)) if grouped else (lambda cp: ls.step(cp, only=layer_ids))
+    per_pass = len([g for g in ls._groups() if all(li in layer_ids for li in g)]) if grouped else len(layer_ids)
     if use_graph:
-        graph = capture_graph(torch, lambda i: ls.step(i % copies, only=layer_ids), copies)
-        per_replay = copies * len(layer_ids)
+        graph = capture_graph(torch, lambda i: step_fn(i % copies), copies)
+        per_replay = copies * per_pass
         n = max(1, launches // per_replay)
         for _ in range(3):
             graph.replay()
         ms = time_events(torch, lambda i: graph.replay(), n)
-        return ms / (n * per_replay)
-    n = max(1, launches // len(layer_ids))
+        return ms / (n * per_replay), per_pass
+    n = max(1, launches // per_pass)
     for i in range(copies):
-        ls.step(i % copies, only=layer_ids)
-    ms = time_events(torch, lambda i: ls.step(i % copies, only=layer_ids), n)
-    return ms / (n * len(layer_ids))
+        step_fn(i % copies)
+    ms = time_events(torch, lambda i: step_fn(i % copies), n)
+    return ms / (n * per_pass), per_pass
 
 
 def main():
@@ -407,7 +420,7 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    grouped = use_graph and not args.no_groups
+    grouped = stage == "decode" and not args.no_groups
     res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local), grouped)
     if world > 1:
         dist.barrier()
@@ -429,11 +442,11 @@ def main():
     # ---- end to end through the public API with host buffers (H2D + forwards + D2H per step)
     e2e_steps = max(8, min(200, steps // 10))
     for i in range(3):
-        ls.step_e2e(i % copies)
+        ls.step_e2e(i % copies, grouped)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for i in range(e2e_steps):
-        ls.step_e2e(i % copies)
+        ls.step_e2e(i % copies, grouped)
     e2e_s = time.perf_counter() - t0
     e2e_s = max_over_ranks(e2e_s, device)
     e2e_value = whole_job_value(units_per_step, e2e_steps, e2e_s * 1e3, world)
@@ -442,8 +455,8 @@ def main():
     if stage == "decode":
         dom_ids = [i for i, l in enumerate(workload.layers) if l.bits == 4] or list(range(len(workload.layers)))
         dom_name = "gemv_kernel<int4, grouped>" if workload.layers[dom_ids[0]].bits == 4 else "gemv_kernel<int8>"
-        dom_ms = dominant_kernel_time(torch, ls, dom_ids, 1200, use_graph)
-        dom_bytes = sum(workload.layers[i].weight_bytes for i in dom_ids) / len(dom_ids)
+        dom_ms, dom_launches = dominant_kernel_time(torch, ls, dom_ids, 1200, use_graph, grouped)
+        dom_bytes = sum(workload.layers[i].weight_bytes for i in dom_ids) / dom_launches
         achieved = dom_bytes / 1e9 / (dom_ms / 1e3)
         roof = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((workload.name, M)),
@@ -452,7 +465,7 @@ def main():
                 "frac_of_nominal_8tbs": achieved / 8000.0}
     else:
         dom_ids = [i for i, l in enumerate(workload.layers) if l.bits == 4] or list(range(len(workload.layers)))
-        dom_ms = dominant_kernel_time(torch, ls, dom_ids, 30 * len(dom_ids), False)
+        dom_ms, _ = dominant_kernel_time(torch, ls, dom_ids, 30 * len(dom_ids), False)
         dom_flops = sum(workload.layers[i].flops(M) for i in dom_ids) / len(dom_ids)
         achieved = dom_flops / 1e12 / (dom_ms / 1e3)
         peak = peaks["bf16_tflops"]
@@ -469,11 +482,11 @@ def main():
         "config": {"workload": workload.name, "M": M, "layers": [f"{l.name}:{l.N}x{l.K}:int{l.bits}" for l in workload.layers],
                    "weight_copies": copies, "weight_bytes_per_step": ls.weight_bytes,
                    "l2": f"{copies} weight copies ({copies * layer_bytes / 1e6:.0f} MB) rotated per step; no flush",
-                   "launch": ("cuda graph + programmatic dependent launch" + (", q/k/v and gate/up as one grouped call each" if grouped else ""))
-                             if use_graph else "stream launches",
+                   "launch": ("cuda graph + programmatic dependent launch" if use_graph else "stream launches")
+                             + (", q/k/v and gate/up as one grouped call each" if grouped else ""),
                    "parallelism": "replicas only" if world > 1 else "single gpu"},
         "clocks": res["clocks"], "gpu_launches": res["launches"],
-        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": ls.h2d_bytes, "d2h_bytes_per_step": ls.d2h_bytes,
+        "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": ls.h2d_bytes(grouped), "d2h_bytes_per_step": ls.d2h_bytes,
                 "steps": e2e_steps},
         "roofline": roof,
         "frac_of_measured_peak": value / world / (peaks["hbm_gbs"] if stage == "decode" else peaks["bf16_tflops"]),
@@ -506,7 +519,7 @@ def prefill_sub(torch, device, peaks, steps, local):
         return {"unavailable": str(e)}
     tf = ls.flops * res["steps"] / 1e12 / (res["ms"] / 1e3)
     dom_ids = [i for i, l in enumerate(w.layers) if l.bits == 4]
-    dom_ms = dominant_kernel_time(torch, ls, dom_ids, 30, False)
+    dom_ms, _ = dominant_kernel_time(torch, ls, dom_ids, 30, False)
     dom_flops = sum(w.layers[i].flops(M) for i in dom_ids) / len(dom_ids)
     ach = dom_flops / 1e12 / (dom_ms / 1e3)
     return {"metric": "prefill_tflops", "value": tf, "unit": "TFLOP/s", "steps": res["steps"],
