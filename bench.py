@@ -420,7 +420,7 @@ def main():
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
-    grouped = stage == "decode" and not args.no_groups
+    grouped = not args.no_groups
     res = bench_stage(torch, ls, stage, args.steps, args.warmup, use_graph, physical_gpu_index(local), grouped)
     if world > 1:
         dist.barrier()
@@ -514,7 +514,7 @@ def prefill_sub(torch, device, peaks, steps, local):
     M = w.Ms[0]
     try:
         ls = LayerSet(w, M, 2, device)
-        res = bench_stage(torch, ls, "prefill", steps, 3, False, physical_gpu_index(local))
+        res = bench_stage(torch, ls, "prefill", steps, 3, False, physical_gpu_index(local), grouped=True)
     except P.QLinearError as e:
         return {"unavailable": str(e)}
     tf = ls.flops * res["steps"] / 1e12 / (res["ms"] / 1e3)

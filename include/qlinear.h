@@ -100,8 +100,10 @@ ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M
  * a launch of their own (the paper's operator fusion, Section 3 "Operator Fusion", merges kernels for
  * the same reason: launch overhead and memory-bound work).  Every output is bit-identical to what
  * qlinear_forward gives for that layer only if the K split chosen for the group equals the layer's own;
- * it always meets the same tolerance, and is run-to-run deterministic.  For larger M the layers run
- * one after the other with the prefill kernel.
+ * it always meets the same tolerance, and is run-to-run deterministic.  For larger M the layers share
+ * one launch of the prefill kernel when every layer qualifies for its CTA-pair form (M > 128 and a
+ * multiple of 256 output channels after padding to 128); the tiles of all layers then fill the
+ * persistent grid together.  Otherwise they run one after the other.
  *   hs      host array of n handles; ys_dev host array of n device pointers (fp16 [M, N_i], 16-byte
  *           aligned, not overlapping x_dev or one another); x_dev as in qlinear_forward.
  * Asynchronous, allocates nothing.  Calls that put the same handle first must not run concurrently

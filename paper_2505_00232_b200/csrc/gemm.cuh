@@ -49,7 +49,16 @@ struct GemmParams {
     int32_t n_whole;                         // pair kernel: units [0, n_whole) are whole tiles, the rest are parts
     float* scratch;                          // pair kernel, split > 1: fp32 partial tiles [tile][part][rank][256][128]
     unsigned int* counters;                  // pair kernel, split > 1: arrivals per (tile, rank, quarter), zero between launches
+    // pair kernel: up to kGemmMaxGroup layers that read the same x in one launch; their row super-blocks are
+    // numbered one after the other, rsb_end[i] = row super-blocks of layers 0..i (each layer an even number)
+    const uint8_t* lbody[4];
+    const __half* lscales[4];
+    __half* ly[4];
+    int32_t lN[4];
+    int32_t rsb_end[4];
+    int32_t n_layers;
 };
+constexpr int kGemmMaxGroup = 4;
 
 struct GemmPlan {
     int32_t dummy;

@@ -61,6 +61,17 @@ __device__ __forceinline__ PairUnit pair_unit(int t, const GemmParams& p)
     return u;
 }
 
+// Row super-block numbered through all layers of the launch -> (layer, row super-block inside it).
+__device__ __forceinline__ int pair_layer(const GemmParams& p, int& rsb)
+{
+    int ly = 0;
+#pragma unroll
+    for (int i = 1; i < kGemmMaxGroup; ++i)
+        if (i < p.n_layers && rsb >= p.rsb_end[i - 1]) ly = i;
+    rsb -= ly ? p.rsb_end[ly - 1] : 0;
+    return ly;
+}
+
 template <int BITS, bool GROUPED, int TB>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
@@ -131,9 +142,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
                 const PairUnit u = pair_unit(t, p);
                 const int tile = u.tile, step0 = u.step0, n_steps = u.nsteps;
-                const int rsb = 2 * (tile / n_mblk) + (int)rank;
+                int rsb = 2 * (tile / n_mblk) + (int)rank;
+                const int ly = pair_layer(p, rsb);
                 const int m0 = (tile % n_mblk) * TILE_N + 128 * (int)rank;   // this CTA's 128 tokens of each token block
-                const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
+                const uint8_t* wsrc = p.lbody[ly] + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
                     QL_GTRACE(0, issued);
@@ -258,24 +270,26 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             const uint32_t use = TB == 1 ? (uint32_t)(j >> 1) : (uint32_t)j;
             const PairUnit u = pair_unit(t, p);
             const int tile = u.tile, part = u.part;
-            const int rsb = 2 * (tile / n_mblk) + (int)rank, m0 = (tile % n_mblk) * TILE_N;
+            int rsb = 2 * (tile / n_mblk) + (int)rank;
+            const int ly = pair_layer(p, rsb);
+            const int m0 = (tile % n_mblk) * TILE_N, N = p.lN[ly];
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
             const int n = rsb * kRsbRows + quarter * 32 + lane;
             float scale = 1.f;
-            if (!GROUPED && n < p.N) scale = __half2float(p.chan_scales[n]);
+            if (!GROUPED && n < N) scale = __half2float(p.lscales[ly][n]);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
-            __half* yrow = p.y + (int64_t)m0 * p.N + n;
+            __half* yrow = p.ly[ly] + (int64_t)m0 * N + n;
             const int m_left = min(TILE_N, p.M - m0);                    // accumulator column = token m0 + column
             if (u.parts == 1) {
 #pragma unroll 1
                 for (int cc = 0; cc < m_left; cc += 16) {
                     uint32_t r[16];
                     tmem_ld16(taddr + (uint32_t)cc, r);
-                    if (n < p.N) {
+                    if (n < N) {
 #pragma unroll
                         for (int q = 0; q < 16; ++q)
-                            if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(__uint_as_float(r[q]) * scale);
+                            if (cc + q < m_left) yrow[(int64_t)(cc + q) * N] = __float2half_rn(__uint_as_float(r[q]) * scale);
                     }
                 }
                 tc_fence_before();
@@ -329,10 +343,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 #pragma unroll
                             for (int q = 0; q < 16; ++q) acc[q] = ((acc[q] + v1[q]) + v2[q]) + v3[q];
                         }
-                        if (n < p.N) {
+                        if (n < N) {
 #pragma unroll
                             for (int q = 0; q < 16; ++q)
-                                if (cc + q < m_left) yrow[(int64_t)(cc + q) * p.N] = __float2half_rn(acc[q] * scale);
+                                if (cc + q < m_left) yrow[(int64_t)(cc + q) * N] = __float2half_rn(acc[q] * scale);
                         }
                     }
                     if (lane == 0) *cnt = 0;                             // ready for the next launch
@@ -370,11 +384,22 @@ inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2
 // A layer can only ever be split if it has few row-super-block pairs.
 inline bool gemm_pair_may_split(const Layout& L, int) { return (L.n_rsb % 2) == 0; }
 
+// The layers of one launch: all read the same x and agree in K and scheme; each has an even number of row
+// super-blocks.  L is the layout of the first one (K, chunking and scheme are taken from it).
+struct GemmPairLayers {
+    int n;
+    const Layout* L[kGemmMaxGroup];
+    const uint8_t* blob[kGemmMaxGroup];
+    void* y[kGemmMaxGroup];
+    int n_rsb() const { int t = 0; for (int i = 0; i < n; ++i) t += L[i]->n_rsb; return t; }
+};
+
 template <int BITS, bool GROUPED, int TB>
-ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st, int device,
+ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device,
                            bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
     using S = GemmPairSmem<BITS, TB>;
+    const Layout& L = *set.L[0];
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return QL_ERR_CUDA;
     CUtensorMap map;
@@ -396,14 +421,22 @@ ql_status gemm_pair_launch(const Layout& L, const uint8_t* blob, const void* x, 
         attr_set[device] = true;
     }
     GemmParams prm{};
-    prm.body = blob + L.body_offset;
-    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(blob + L.chan_scale_offset);
-    prm.y = static_cast<__half*>(y);
+    int n_rsb = 0;
+    for (int i = 0; i < set.n; ++i) {
+        const Layout& Li = *set.L[i];
+        prm.lbody[i] = set.blob[i] + Li.body_offset;
+        prm.lscales[i] = Li.grouped ? nullptr : reinterpret_cast<const __half*>(set.blob[i] + Li.chan_scale_offset);
+        prm.ly[i] = static_cast<__half*>(set.y[i]);
+        prm.lN[i] = Li.N;
+        n_rsb += Li.n_rsb;
+        prm.rsb_end[i] = n_rsb;
+    }
+    prm.n_layers = set.n;
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
-    prm.n_rsb = L.n_rsb;
-    const int tiles = (L.n_rsb / 2) * ((M + 256 * TB - 1) / (256 * TB));
+    prm.n_rsb = n_rsb;
+    const int tiles = (n_rsb / 2) * ((M + 256 * TB - 1) / (256 * TB));
     // whole tiles fill the full rounds of the persistent grid; the tiles of the last partial round are split
     const int clusters = num_sms / 2;
     // (splitting the tail of a multi-round schedule was measured and does not pay: the exposed scratch
@@ -445,28 +478,29 @@ inline bool gemm_pair_applicable(const Layout& L, int M)
     return (L.n_rsb % 2) == 0 && M > 128;
 }
 
-inline ql_status gemm_pair_forward(const Layout& L, const uint8_t* blob, const void* x, void* y, int M, cudaStream_t st,
+inline ql_status gemm_pair_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st,
                                    int device, bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
     // Token blocks per tile: a step of a 512-token tile costs two steps of a 256-token tile (the kernel is
     // bound by the tensor pipe and its operand traffic, not by dequantisation), so the wider tile only pays
     // where it saves rounds of the persistent grid.
+    const Layout& L = *set.L[0];
     const char* f = std::getenv("QLINEAR_GEMM_TB");
     int tb = (f && *f) ? std::atoi(f) : 0;
     if (tb == 0) {
-        const int clusters = num_sms / 2, pairs = L.n_rsb / 2;
+        const int clusters = num_sms / 2, pairs = set.n_rsb() / 2;
         const int tiles1 = pairs * ((M + 255) / 256), tiles2 = pairs * ((M + 511) / 512);
         const int rounds1 = (tiles1 + clusters - 1) / clusters, rounds2 = (tiles2 + clusters - 1) / clusters;
         tb = (tiles1 >= clusters && 2 * rounds2 <= rounds1) ? 2 : 1;
     }
     if (tb == 2 && M > 256) {
-        if (L.bits == 8) return gemm_pair_launch<8, false, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-        if (L.grouped) return gemm_pair_launch<4, true, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-        return gemm_pair_launch<4, false, 2>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+        if (L.bits == 8) return gemm_pair_launch<8, false, 2>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+        if (L.grouped) return gemm_pair_launch<4, true, 2>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+        return gemm_pair_launch<4, false, 2>(set, x, M, st, device, pdl, num_sms, scratch, counters);
     }
-    if (L.bits == 8) return gemm_pair_launch<8, false, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-    if (L.grouped) return gemm_pair_launch<4, true, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
-    return gemm_pair_launch<4, false, 1>(L, blob, x, y, M, st, device, pdl, num_sms, scratch, counters);
+    if (L.bits == 8) return gemm_pair_launch<8, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+    if (L.grouped) return gemm_pair_launch<4, true, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+    return gemm_pair_launch<4, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
 }
 
 }  // namespace ql

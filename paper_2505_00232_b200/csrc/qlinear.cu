@@ -356,8 +356,11 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
-    if (gemm_pair_applicable(h->L, M))
-        return gemm_pair_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms, h->gemm_scratch, h->gemm_counters);
+    if (gemm_pair_applicable(h->L, M)) {
+        GemmPairLayers set{};
+        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y;
+        return gemm_pair_forward(set, x, M, st, h->device, h->pdl, h->num_sms, h->gemm_scratch, h->gemm_counters);
+    }
     return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
@@ -376,6 +379,19 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         DeviceGuard guard(hs[0]->device);
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
         return forward_gemv(const_cast<qlinear_s* const*>(hs), n, x, ys, M, static_cast<cudaStream_t>(stream));
+    }
+    if (n > 1 && M > hs[0]->gemv_max_m) {                                // prefill: one launch of the CTA-pair kernel
+        bool pair_ok = true;
+        for (int i = 0; i < n; ++i) pair_ok = pair_ok && gemm_pair_applicable(hs[i]->L, M);
+        if (pair_ok) {
+            DeviceGuard guard(hs[0]->device);
+            if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+            GemmPairLayers set{};
+            set.n = n;
+            for (int i = 0; i < n; ++i) { set.L[i] = &hs[i]->L; set.blob[i] = hs[i]->blob; set.y[i] = ys[i]; }
+            return gemm_pair_forward(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
+                                     hs[0]->gemm_scratch, hs[0]->gemm_counters);
+        }
     }
     for (int i = 0; i < n; ++i) {
         ql_status s = qlinear_forward(hs[i], x, ys[i], M, stream);

@@ -166,3 +166,28 @@ def test_lm_head_decode_config5b(P, torch):
         y64[:, r0:r1], A[:, r0:r1], _ = O.linear(x, q[r0:r1], s[r0:r1], layer.group)
     ok, rel, worst = O.check_against(y, y64, A)
     assert ok, (rel, worst)
+
+
+GROUPS = [
+    # (M, K, bits, group, [N_i]): one launch of the CTA-pair kernel for layers that share x
+    (300, 512, 8, 0, [512, 256, 256]),           # q/k/v-like; few tiles: split along K
+    (200, 1024, 4, 32, [200, 256]),              # ragged N, ragged M
+    (1024, 256, 8, 0, [2560, 1280, 1024]),       # enough tiles for 512-token tiles
+    (640, 384, 4, 0, [512, 768]),                # int4 per channel
+]
+
+
+@pytest.mark.parametrize("M,K,bits,group,Ns", GROUPS)
+def test_forward_group_prefill_parity(P, torch, M, K, bits, group, Ns):
+    cases = [rand_case(8000 + 13 * i + N + K, M, N, K, bits, group) for i, N in enumerate(Ns)]
+    x = cases[0][2]
+    lins = [P.QLinear.from_weights(q, s, bits, group, device="cuda:0") for q, s, _ in cases]
+    xd = torch.from_numpy(x).cuda()
+    ys = P.qlinear_forward_group(lins, xd)
+    torch.cuda.synchronize()
+    assert lins[0].device_status()[0] == 0
+    for (q, s, _), y in zip(cases, ys):
+        assert_parity(y.cpu().numpy(), x, q, s, group)
+    again = P.qlinear_forward_group(lins, xd)
+    for a, b in zip(ys, again):
+        assert torch.equal(a, b)
