@@ -228,3 +228,19 @@ def test_forward_group_prefill_and_errors(P, torch):
         P.qlinear_forward_group([lins[0], other], xd)
     with pytest.raises(P.QLinearError):
         P.qlinear_forward_group(lins * 3, xd)            # more than four layers
+
+
+@pytest.mark.parametrize("wi,names,M", [(2, ("q", "k", "v"), 1), (2, ("gate", "up"), 1), (2, ("gate", "up"), 4),
+                                        (1, ("q", "k", "v"), 1), (1, ("gate", "up"), 1)])
+def test_forward_group_configs_full_size(P, torch, wi, names, M):
+    """The grouped launches bench.py times (configs 2 and 3 at full size) against the oracle, layer by layer."""
+    w = C.CONFIGS[wi]
+    ids = [i for i, l in enumerate(w.layers) if l.name in names]
+    ws = [C.layer_weights(w.seed, w.layers[i], i) for i in ids]
+    x = C.layer_activations(w.seed, w.layers[ids[0]], M, ids[0])
+    lins = [P.QLinear.from_weights(q, s, w.layers[i].bits, w.layers[i].group, device="cuda:0") for i, (q, s) in zip(ids, ws)]
+    ys = P.qlinear_forward_group(lins, torch.from_numpy(x).cuda())
+    torch.cuda.synchronize()
+    assert lins[0].device_status()[0] == 0
+    for i, (q, s), y in zip(ids, ws, ys):
+        assert_parity(y.cpu().numpy(), x, q, s, w.layers[i].group)

@@ -191,3 +191,26 @@ def test_forward_group_prefill_parity(P, torch, M, K, bits, group, Ns):
     again = P.qlinear_forward_group(lins, xd)
     for a, b in zip(ys, again):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("names", [("q", "k", "v"), ("gate", "up")], ids=["qkv", "gate_up"])
+def test_forward_group_config5_llama_prefill_sampled_columns(P, torch, names):
+    """The grouped prefill launches bench.py times (config 5, M = 2048): all tokens of 512 seeded output
+    channels per layer (plus the first and last 16) against the oracle."""
+    w = C.CONFIGS[4]
+    M = w.Ms[0]
+    ids = [i for i, l in enumerate(w.layers) if l.name in names]
+    ws = [C.layer_weights(w.seed, w.layers[i], i) for i in ids]
+    x = C.layer_activations(w.seed, w.layers[ids[0]], M, ids[0])
+    lins = [P.QLinear.from_weights(q, s, w.layers[i].bits, w.layers[i].group, device="cuda:0") for i, (q, s) in zip(ids, ws)]
+    ys = P.qlinear_forward_group(lins, torch.from_numpy(x).cuda())
+    torch.cuda.synchronize()
+    assert lins[0].device_status()[0] == 0
+    for i, (q, s), y in zip(ids, ws, ys):
+        layer = w.layers[i]
+        y = y.cpu().numpy()
+        rng = np.random.default_rng(100 + i)
+        cols = np.unique(np.concatenate([np.arange(16), np.arange(layer.N - 16, layer.N),
+                                         rng.choice(layer.N, size=512, replace=False)]))
+        assert_parity(y[:, cols], x, q[cols], s[cols], layer.group)
+        assert np.isfinite(y.astype(np.float32)).all()
