@@ -112,6 +112,17 @@ ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
 
+/* Embedding lookup from a quantised table (Section 4.2: the mixed 8/4/4 scheme keeps the embedding table
+ * in int4 like the feed-forward weights).  The handle's layer is read as a table of N rows of K values:
+ *   y_dev[t, k] = fp16( s[ids[t], k / group] * q[ids[t], k] )      for t in [0, n), k in [0, K)
+ * the correctly rounded product (one rounding), i.e. the dequantised row, bit for bit.  The same blob can
+ * serve as LM head through qlinear_forward.
+ *   ids_dev  device, int32 [n], 4-byte aligned; a row number outside [0, N) gives a row of zeros
+ *   y_dev    device, fp16 [n, K] row-major contiguous, 16-byte aligned
+ * Asynchronous on `cuda_stream`, allocates nothing.  n == 0 is a no-op (the pointers are not looked at).
+ * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, n < 0), QL_ERR_CUDA (launch failure). */
+ql_status qlinear_embed(qlinear_t h, const int32_t* ids_dev, int32_t n, void* y_dev, void* cuda_stream);
+
 /* The kernel qlinear_forward uses for M tokens on this handle (0 if h is NULL or M < 1). */
 int32_t qlinear_path_for(qlinear_t h, int32_t M);
 

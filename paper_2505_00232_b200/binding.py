@@ -20,7 +20,7 @@ QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ALLOC, QL_ERR_CUDA, QL_ERR_DEVICE
 QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_embed",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version",
 )
@@ -60,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_debug_unpack_device.restype = ctypes.c_int
     lib.qlinear_forward_group.argtypes = [ctypes.POINTER(vp), ctypes.c_int32, vp, ctypes.POINTER(vp), ctypes.c_int32, vp]
     lib.qlinear_forward_group.restype = ctypes.c_int
+    lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
+    lib.qlinear_embed.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.qlinear_device_status.restype = ctypes.c_int
     lib.qlinear_decode_static.argtypes = [dp, vp, vp, vp, i32, ctypes.c_int, vp]
@@ -218,6 +220,20 @@ class QLinear:
     def forward_raw(self, x_ptr: int, y_ptr: int, M: int, stream=None) -> None:
         _check(lib.qlinear_forward(self._h, ctypes.c_void_p(x_ptr), ctypes.c_void_p(y_ptr), M, _stream_ptr(stream)),
                "qlinear_forward")
+
+    def embed(self, ids, out=None, stream=None):
+        """ids: int32 CUDA tensor [n] -> fp16 [n, K], the dequantised rows ids of the table (qlinear_embed)."""
+        import torch
+        if ids.dim() != 1 or ids.dtype != torch.int32 or not ids.is_cuda or not ids.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_embed (ids must be a contiguous int32 CUDA vector)")
+        n = ids.shape[0]
+        if out is None:
+            out = torch.empty((n, self.desc.K), dtype=torch.float16, device=ids.device)
+        elif out.shape != (n, self.desc.K) or out.dtype != torch.float16 or not out.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_embed (bad out tensor)")
+        _check(lib.qlinear_embed(self._h, ctypes.c_void_p(ids.data_ptr()), n, ctypes.c_void_p(out.data_ptr()),
+                                 _stream_ptr(stream)), "qlinear_embed")
+        return out
 
     def path_for(self, M: int) -> int:
         return int(lib.qlinear_path_for(self._h, M))

@@ -19,6 +19,7 @@ __device__ unsigned int g_device_flag[2];
 }  // namespace ql
 
 #include "dequant.cuh"
+#include "embed.cuh"
 #include "gemv.cuh"
 #include "gemv_stream.cuh"
 #include "gemm.cuh"
@@ -398,6 +399,28 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         if (s != QL_OK) return s;
     }
     return QL_OK;
+}
+
+extern "C" ql_status qlinear_embed(qlinear_t h, const int32_t* ids, int32_t n, void* y, void* stream)
+{
+    if (!h || n < 0) return QL_ERR_INVALID_ARG;
+    if (n == 0) return QL_OK;                                            // nothing to do: the pointers may be null
+    if (!ids || !y) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(y) & 15) || (reinterpret_cast<uintptr_t>(ids) & 3)) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    const Layout& L = h->L;
+    EmbedParams prm{};
+    prm.body = h->blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
+    prm.ids = ids;
+    prm.y = static_cast<__half*>(y);
+    prm.n = n; prm.N = L.N; prm.K = L.K; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (L.bits == 8) embed_kernel<8, false><<<n, 128, 0, st>>>(prm);
+    else if (L.grouped) embed_kernel<4, true><<<n, 128, 0, st>>>(prm);
+    else embed_kernel<4, false><<<n, 128, 0, st>>>(prm);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
 extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, void* stream)

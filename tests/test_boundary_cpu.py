@@ -129,6 +129,7 @@ def test_host_calls_that_need_no_device(P):
     assert P.lib.qlinear_create(ctypes.byref(bad), ctypes.c_void_p(256), 0, ctypes.byref(h)) == 2
     assert P.lib.qlinear_create(ctypes.byref(d), ctypes.c_void_p(260), 0, ctypes.byref(h)) == 1  # misaligned
     assert P.lib.qlinear_forward(None, ctypes.c_void_p(16), ctypes.c_void_p(32), 1, None) == 1
+    assert P.lib.qlinear_embed(None, ctypes.c_void_p(16), 1, ctypes.c_void_p(32), None) == 1
     # grouped call: null arrays, n outside 1..4 and null handles are refused before any CUDA call
     hs = (ctypes.c_void_p * 2)(None, None)
     ys = (ctypes.c_void_p * 2)(ctypes.c_void_p(32), ctypes.c_void_p(64))
