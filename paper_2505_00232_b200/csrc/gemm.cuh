@@ -9,7 +9,7 @@
 // runs under the main loop of the next.  Per CTA:
 //
 //   warp 0        producer: one bulk copy of the packed weight block(s) of the k-step (contiguous in
-//                 the blob) and one TMA tile load of x [BN tokens x 64 k] (128-byte swizzle, no multicast)
+//                 the blob) and one TMA tile load of x [BN tokens x 64 k] (128-byte swizzle; every CTA loads for itself)
 //   warps 2..17   dequantise: packed block (shared) -> registers -> exact fp16 integers (x group scale
 //                 for grouped int4) -> the K-major 128-byte-swizzled A tile in shared memory
 //   warp 1        issues tcgen05.mma (A, B from shared memory, fp32 accumulator in tensor memory),

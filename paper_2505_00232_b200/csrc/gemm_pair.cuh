@@ -4,12 +4,12 @@
 // the x traffic from L2 and the shared-memory operand reads per flop are half of the single-CTA kernel's
 // (paper Section 3.7: the prefill stage is compute-bound; the point here is to keep it that way).
 //
-// Roles per CTA are those of gemm.cuh.  Cross-CTA protocol (no TMA multicast anywhere):
+// Roles per CTA are those of gemm.cuh.  Cross-CTA protocol (every CTA issues its own loads; nothing is loaded for a peer):
 //   * dequantise warps arrive on their own CTA's afull barrier (a warp dequantises only after its CTA's
 //     TMA data landed, so "A tile written" implies "x half landed"); in the peer CTA the otherwise idle
 //     MMA warp relays each completed afull phase to the leader with ONE remote arrive, on the leader's
 //     afull barrier (17 arrivals there: its own 16 warps and the relay);
-//   * the leader's tcgen05.commit signals the empty / tfull barriers of BOTH CTAs (commit multicast);
+//   * the leader's tcgen05.commit signals the empty / tfull barriers of BOTH CTAs (cluster mask 3 on the commit);
 //   * the epilogue warps of both CTAs arrive on the leader's tempty barrier (8 arrivals);
 //   * cluster barriers bracket the kernel so that no CTA exits while its peer can still touch it.
 #pragma once
