@@ -131,6 +131,12 @@ int32_t qlinear_path_for(qlinear_t h, int32_t M);
  * exactly the integers that were packed.  Asynchronous on `cuda_stream`. */
 ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_dev_out, void* cuda_stream);
 
+/* Test aid for the failure path: launches a one-warp kernel that runs the kernels' bounded wait on a
+ * barrier nothing ever completes.  The wait gives up after about a second, records its code (0x9A0) and
+ * the kernel returns normally; the next qlinear_device_status reports QL_ERR_DEVICE_TIMEOUT with that code
+ * and the device stays usable.  Asynchronous on `cuda_stream`. */
+ql_status qlinear_debug_expire_wait(qlinear_t h, void* cuda_stream);
+
 /* Synchronises the handle's device and reports whether any kernel launched through it gave up a
  * bounded wait (QL_ERR_DEVICE_TIMEOUT), else QL_OK.  `detail`, if not NULL, receives a code that
  * identifies the wait.  Clears the condition. */

@@ -21,7 +21,7 @@ QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
 
 EXPORTS = (
     "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_embed",
-    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
+    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version",
 )
 
@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_forward_group.restype = ctypes.c_int
     lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
     lib.qlinear_embed.restype = ctypes.c_int
+    lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
+    lib.qlinear_debug_expire_wait.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.qlinear_device_status.restype = ctypes.c_int
     lib.qlinear_decode_static.argtypes = [dp, vp, vp, vp, i32, ctypes.c_int, vp]
@@ -244,6 +246,10 @@ class QLinear:
         _check(lib.qlinear_debug_unpack_device(self._h, ctypes.c_void_p(q.data_ptr()), _stream_ptr(stream)),
                "qlinear_debug_unpack_device")
         return q
+
+    def debug_expire_wait(self, stream=None) -> None:
+        """Runs the kernels' bounded wait on a barrier nothing completes (about a second); see device_status."""
+        _check(lib.qlinear_debug_expire_wait(self._h, _stream_ptr(stream)), "qlinear_debug_expire_wait")
 
     def device_status(self):
         detail = ctypes.c_uint32(0)

@@ -267,6 +267,20 @@ __global__ void __launch_bounds__(256) debug_unpack_kernel(const uint8_t* body, 
     }
 }
 
+// Test aid: the bounded wait of the kernels on a barrier that nothing completes.
+__global__ void __launch_bounds__(32) expire_wait_kernel()
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ volatile uint32_t abort_word;
+    if (threadIdx.x == 0) {
+        abort_word = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) mbar_wait<true>(smem_u32(&bar), 0, &abort_word, 0x9A0);   // gives up, records the code
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -547,6 +561,15 @@ extern "C" ql_status qlinear_decode_static(const qlinear_desc* d, const void* pa
     else e = launch_stream_static<4, false>(prm, st, device);
     if (e != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
     return QL_OK;
+}
+
+extern "C" ql_status qlinear_debug_expire_wait(qlinear_t h, void* stream)
+{
+    if (!h) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
 extern "C" ql_status qlinear_device_status(qlinear_t h, uint32_t* detail)
