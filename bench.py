@@ -478,7 +478,7 @@ def main():
     line = {
         "metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": steps, "warmup": args.warmup,
         "ms_per_step": res["ms"] / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 x int4/int8 -> f32 accumulate", "data": "synthetic",
+        "dtype": "f16", "dtype_detail": "int4/int8 weights unpacked to f16, f16 activations, f32 accumulate", "data": "synthetic",
         "config": {"workload": workload.name, "M": M, "layers": [f"{l.name}:{l.N}x{l.K}:int{l.bits}" for l in workload.layers],
                    "weight_copies": copies, "weight_bytes_per_step": ls.weight_bytes,
                    "l2": f"{copies} weight copies ({copies * layer_bytes / 1e6:.0f} MB) rotated per step; no flush",
