@@ -35,8 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum, one ncu
-# capture each; figures and commands in profiles/decode_gemv_int4_llama_gate_up_full.md and
-# profiles/prefill_gemm_pair_int4_llama_ffn_full.md), averaged over the launches bench.py times.
+# capture each, summarised with its command under profiles/), averaged over the launches this file times.
 NCU_TRAFFIC_BYTES = {
     ("llama31_8b_decode", 1): (66.095104e6 + 0.455936e6 + 33.085440e6) / 2,     # gate+up and down launches
     ("llama31_8b_prefill", 2048): (73.6e6 + 73.6e6 + 95.9e6) / 3,            # gate, up, down (reads + y write-back)
