@@ -213,7 +213,8 @@ def test_forward_group_parity(P, torch, M, K, bits, group, Ns):
 
 
 def test_forward_group_prefill_and_errors(P, torch):
-    """M > 8 runs the layers one after the other (same results as single calls); mismatched layers are refused."""
+    """M > 8 with layers the CTA-pair prefill kernel does not take (M <= 128) runs them one after the other (same
+    results as single calls); mismatched layers are refused."""
     M, K = 24, 256
     cases = [rand_case(6000 + N, M, N, K, 4, 32) for N in (128, 264)]
     x = cases[0][2]

@@ -36,6 +36,28 @@ def assert_parity(y_gpu, x, q, s, group):
     assert ok, f"rel_l2={rel:.3e} (tol {O.REL_L2_TOL}) worst |dy|/A={worst:.3e} (tol {O.ELEM_TOL})"
 
 
+def assert_parity_whole_output(y_gpu, x, q, s, group, rows=2048):
+    """Every element of the M x N output against the oracle, walking N in blocks of `rows` output channels
+    (bounds the oracle's fp64 working set).  The relative L2 error is taken over the whole output: squared
+    norms are accumulated across the blocks; the per-element ratio is the maximum over all of them."""
+    N = q.shape[0]
+    d2 = y2 = 0.0
+    worst = 0.0
+    for r0 in range(0, N, rows):
+        r1 = min(N, r0 + rows)
+        y64, A, _ = O.linear(x, q[r0:r1], s[r0:r1], group)
+        d = y_gpu[:, r0:r1].astype(np.float64) - y64
+        d2 += float((d * d).sum())
+        y2 += float((y64 * y64).sum())
+        with np.errstate(divide="ignore", invalid="ignore"):
+            ratio = np.where(A > 0, np.abs(d) / A, np.where(d == 0, 0.0, np.inf))
+        worst = max(worst, float(ratio.max(initial=0.0)))
+    rel = (d2 / y2) ** 0.5 if y2 > 0 else d2 ** 0.5
+    assert rel <= O.REL_L2_TOL and worst <= O.ELEM_TOL, \
+        f"rel_l2={rel:.3e} (tol {O.REL_L2_TOL}) worst |dy|/A={worst:.3e} (tol {O.ELEM_TOL})"
+    assert np.isfinite(y_gpu.astype(np.float32)).all()
+
+
 def rand_case(seed, M, N, K, bits, group):
     layer = C.LayerSpec("t", N, K, bits, group, *((-8, 7) if bits == 4 else (-128, 127)))
     q, s = C.layer_weights(seed, layer)
@@ -134,21 +156,16 @@ def test_parity_config4_gemma_prefill_full(P, torch, li):
 
 
 @pytest.mark.parametrize("li", range(7), ids=[l.name for l in C.LLAMA31_8B])
-def test_parity_config5_llama_prefill_sampled_columns(P, torch, li):
-    """Config 5 at full size (M = 2048), in the launch configuration the bench times.  The oracle
-    checks all 2048 tokens of 512 seeded output channels per layer (plus the first and last 16),
-    and the relative L2 error over that sample."""
+def test_parity_config5_llama_prefill_full(P, torch, li):
+    """Config 5 at full size (M = 2048), in the launch configuration the bench times: every one of the
+    2048 x N outputs of every layer against the oracle."""
     w = C.CONFIGS[4]
     layer, M = w.layers[li], w.Ms[0]
     q, s = C.layer_weights(w.seed, layer, li)
     x = C.layer_activations(w.seed, layer, M, li)
     lin = P.QLinear.from_weights(q, s, layer.bits, layer.group, device="cuda:0")
     y = forward(P, torch, lin, x)
-    rng = np.random.default_rng(li)
-    cols = np.unique(np.concatenate([np.arange(16), np.arange(layer.N - 16, layer.N),
-                                     rng.choice(layer.N, size=512, replace=False)]))
-    assert_parity(y[:, cols], x, q[cols], s[cols], layer.group)
-    assert np.isfinite(y.astype(np.float32)).all()
+    assert_parity_whole_output(y, x, q, s, layer.group)
 
 
 def test_lm_head_decode_config5b(P, torch):
@@ -194,9 +211,9 @@ def test_forward_group_prefill_parity(P, torch, M, K, bits, group, Ns):
 
 
 @pytest.mark.parametrize("names", [("q", "k", "v"), ("gate", "up")], ids=["qkv", "gate_up"])
-def test_forward_group_config5_llama_prefill_sampled_columns(P, torch, names):
-    """The grouped prefill launches bench.py times (config 5, M = 2048): all tokens of 512 seeded output
-    channels per layer (plus the first and last 16) against the oracle."""
+def test_forward_group_config5_llama_prefill_full(P, torch, names):
+    """The grouped prefill launches bench.py times (config 5, M = 2048): every output element of every
+    layer of the group against the oracle."""
     w = C.CONFIGS[4]
     M = w.Ms[0]
     ids = [i for i, l in enumerate(w.layers) if l.name in names]
@@ -207,10 +224,4 @@ def test_forward_group_config5_llama_prefill_sampled_columns(P, torch, names):
     torch.cuda.synchronize()
     assert lins[0].device_status()[0] == 0
     for i, (q, s), y in zip(ids, ws, ys):
-        layer = w.layers[i]
-        y = y.cpu().numpy()
-        rng = np.random.default_rng(100 + i)
-        cols = np.unique(np.concatenate([np.arange(16), np.arange(layer.N - 16, layer.N),
-                                         rng.choice(layer.N, size=512, replace=False)]))
-        assert_parity(y[:, cols], x, q[cols], s[cols], layer.group)
-        assert np.isfinite(y.astype(np.float32)).all()
+        assert_parity_whole_output(y.cpu().numpy(), x, q, s, w.layers[i].group)
