@@ -17,8 +17,26 @@
  * reading the same resident weights.  Quantisation schemes: Section 4.2 (q8 =
  * int8 per channel; 8/4/4 = int8 attention, int4 feed-forward/embedding).
  *
- * All functions are thread-safe; a handle is immutable after creation.  No
- * function falls back to the CPU: without an sm_100 device qlinear_create
+ * Threads and streams.  A handle is immutable after qlinear_create, so any
+ * number of host threads may call the forward functions on it.  The kernels of
+ * two calls may overlap on the GPU (different streams) unless one of them is a
+ * prefill call the library splits along K (a layer, or group of layers, with
+ * fewer 256 x 256 output tiles than half the SM count): those calls meet in one
+ * per-device scratch area and must be ordered against each other by the caller
+ * (same stream, or events).  qlinear_decode_static has its own rule, stated
+ * there.
+ *
+ * Device memory.  The caller owns the packed weights, x and y.  The library
+ * owns one small set of buffers PER DEVICE, allocated when the first handle on
+ * that device is created and kept until the process exits: about 19 MB of fp32
+ * partial tiles plus counters for the K-split prefill case, and one word of
+ * pinned host memory through which kernels report an expired wait.  A handle
+ * itself owns host memory only.
+ *
+ * Environment.  Every QLINEAR_* variable is read once per process, at the
+ * first call that creates a handle; later changes are not seen.
+ *
+ * No function falls back to the CPU: without an sm_100 device qlinear_create
  * fails with QL_ERR_ARCH.
  */
 #ifndef QLINEAR_H
@@ -77,9 +95,10 @@ ql_status qlinear_unpack(const qlinear_desc* desc, const void* packed, int8_t* q
  *   packed_dev  device pointer, 256-byte aligned, qlinear_packed_size(desc) bytes, owned by the caller,
  *               must stay alive and unchanged until qlinear_destroy.
  *   device      CUDA device ordinal that owns packed_dev.
- * The handle owns host memory and a small device scratch (a few MB of partial-sum slots for the streaming
- * decode kernel, allocated here, freed by qlinear_destroy); calls on one handle must be stream-ordered.
- * Errors: QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ARCH
+ * The handle owns host memory only (shape, kernel plans); the first handle on a device also creates that
+ * device's shared buffers (see "Device memory" above), so the first create on a device should come before
+ * any stream capture.
+ * Errors: QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED (descriptor, or a shape no decode plan fits), QL_ERR_ARCH
  * (device is not sm_100), QL_ERR_CUDA, QL_ERR_ALLOC. */
 ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int device, qlinear_t* out);
 
@@ -89,8 +108,10 @@ ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int d
  * Asynchronous: returns after the launch; allocates nothing; never synchronises.  M <= 8 runs the
  * decode kernel, larger M the prefill kernel (Section 3.7); see qlinear_path_for.
  * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, M < 1, M*K or M*N beyond 2^31-1 elements),
- * QL_ERR_CUDA (launch failure, reported synchronously), QL_ERR_DEVICE_TIMEOUT (a previous call on this
- * handle hit a bounded wait; see qlinear_device_status). */
+ * QL_ERR_CUDA (launch failure, reported synchronously), QL_ERR_DEVICE_TIMEOUT (an earlier kernel of this
+ * library on the handle's DEVICE gave up a bounded wait: its output is invalid; nothing is launched, and every
+ * forward call on that device keeps returning this code until qlinear_device_status has cleared it.  The
+ * code reaches the host through pinned memory, so this check costs no synchronisation). */
 ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
 
 /* The same result as n calls of qlinear_forward with one x: ys_dev[i] = x . W_i^T for the n layers hs[i]
@@ -106,8 +127,7 @@ ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M
  * persistent grid together.  Otherwise they run one after the other.
  *   hs      host array of n handles; ys_dev host array of n device pointers (fp16 [M, N_i], 16-byte
  *           aligned, not overlapping x_dev or one another); x_dev as in qlinear_forward.
- * Asynchronous, allocates nothing.  Calls that put the same handle first must not run concurrently
- * from different host threads (the plan of the group is cached in it).
+ * Asynchronous, allocates nothing; the plan of the group is made per call and nothing is written to a handle.
  * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..4 or layers that do not agree. */
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
@@ -137,9 +157,12 @@ ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_dev_out, void* cuda
  * and the device stays usable.  Asynchronous on `cuda_stream`. */
 ql_status qlinear_debug_expire_wait(qlinear_t h, void* cuda_stream);
 
-/* Synchronises the handle's device and reports whether any kernel launched through it gave up a
+/* Synchronises the handle's device and reports whether any kernel of this library on that device gave up a
  * bounded wait (QL_ERR_DEVICE_TIMEOUT), else QL_OK.  `detail`, if not NULL, receives a code that
- * identifies the wait.  Clears the condition. */
+ * identifies the wait.  Clears the condition (the flag the forward calls look at, and the arrival counters
+ * an abandoned K-split launch may have left behind), after which the device's handles work again.
+ * A wait only counts time after the kernel's own stream dependency has resolved: a long-running earlier
+ * kernel in the stream does not expire the waits of the kernel queued behind it. */
 ql_status qlinear_device_status(qlinear_t h, uint32_t* detail);
 
 /* Decode call for callers that cannot allocate device memory.  (The paper has no counterpart: this is
@@ -170,7 +193,7 @@ ql_status qlinear_device_status(qlinear_t h, uint32_t* detail);
 ql_status qlinear_decode_static(const qlinear_desc* desc, const void* packed_dev, const void* x_dev, void* y_dev,
                                 int32_t M, int device, void* cuda_stream);
 
-/* Frees the handle's host memory and its device scratch.  Does not touch the packed blob.  NULL is allowed. */
+/* Frees the handle's host memory.  Does not touch the packed blob or the device's shared buffers.  NULL is allowed. */
 ql_status qlinear_destroy(qlinear_t h);
 
 /* Static, NUL-terminated description of a status code. */
@@ -178,6 +201,14 @@ const char* qlinear_status_string(ql_status s);
 
 /* Library ABI version (major << 16 | minor). */
 uint32_t qlinear_version(void);
+
+/* Test aids (no paper counterpart).  qlinear_debug_plan writes up to n_out of the decode plan's numbers for M
+ * tokens {kernel (1 cluster, 3 streaming), grid CTAs, CTAs per cluster, K slices per CTA, chunks per slice,
+ * 1000 x (work of the busiest SM / mean), row-blocks, chunks along K} and returns how many it wrote (0 on bad
+ * arguments).  qlinear_debug_config_reads returns how many times the QLINEAR_* environment has been read by
+ * this process (1 after the first call, for good). */
+int32_t qlinear_debug_plan(qlinear_t h, int32_t M, int32_t* out, int32_t n_out);
+uint32_t qlinear_debug_config_reads(void);
 
 #ifdef __cplusplus
 }

@@ -22,7 +22,7 @@ QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
 EXPORTS = (
     "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_embed",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
-    "qlinear_status_string", "qlinear_version",
+    "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
 
 
@@ -73,6 +73,9 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_status_string.argtypes = [ctypes.c_int]
     lib.qlinear_status_string.restype = ctypes.c_char_p
     lib.qlinear_version.restype = ctypes.c_uint32
+    lib.qlinear_debug_plan.argtypes = [vp, i32, ctypes.POINTER(i32), i32]
+    lib.qlinear_debug_plan.restype = i32
+    lib.qlinear_debug_config_reads.restype = ctypes.c_uint32
     return lib
 
 
@@ -148,9 +151,16 @@ def qlinear_decode_static(desc: Desc, packed, x, out=None, stream=None):
     """Decode (M <= 8) without a handle and without any allocation inside the library: the caller passes the
     packed device tensor, x and (optionally) the output tensor; see include/qlinear.h."""
     import torch
+    if (x.dim() != 2 or x.shape[1] != desc.K or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous()):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_decode_static (x must be contiguous fp16 CUDA [M, K])")
+    if (not packed.is_cuda or packed.dtype != torch.uint8 or not packed.is_contiguous()
+            or packed.numel() < qlinear_packed_size(desc) or packed.device != x.device):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_decode_static (packed must be a contiguous uint8 CUDA tensor of the packed size)")
     M = x.shape[0]
     if out is None:
         out = torch.empty((M, desc.N), dtype=torch.float16, device=x.device)
+    elif out.shape != (M, desc.N) or out.dtype != torch.float16 or not out.is_contiguous() or out.device != x.device:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_decode_static (bad out tensor)")
     _check(lib.qlinear_decode_static(ctypes.byref(desc.c()), ctypes.c_void_p(packed.data_ptr()),
                                      ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(out.data_ptr()), M,
                                      x.device.index or 0, _stream_ptr(stream)), "qlinear_decode_static")

@@ -24,6 +24,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "../../include/qlinear.h"
 #include "dequant.cuh"
 #include "layout.h"
@@ -59,31 +62,6 @@ struct GemmParams {
     int32_t n_layers;
 };
 constexpr int kGemmMaxGroup = 4;
-
-struct GemmPlan {
-    int32_t dummy;
-};
-
-#ifdef QL_TRACE
-// Developer aid (not compiled by default): %globaltimer stamps of the first k-steps of CTAs 0 and 1.
-constexpr int kGTraceSteps = 48, kGTraceEvents = 8;
-__device__ unsigned long long g_gemm_trace[2][kGTraceEvents][kGTraceSteps];
-#ifndef QL_TRACE_OFFSET
-#define QL_TRACE_OFFSET 0
-#endif
-__device__ __forceinline__ void gemm_trace(int ev, int step)
-{
-    step -= QL_TRACE_OFFSET;                                             // first recorded k-step of the CTA
-    if (blockIdx.x < 2 && step >= 0 && step < kGTraceSteps) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        g_gemm_trace[blockIdx.x][ev][step] = t;
-    }
-}
-#define QL_GTRACE(ev, step) gemm_trace(ev, step)
-#else
-#define QL_GTRACE(ev, step) do { } while (0)
-#endif
 
 // Per-lane constants and the per-step work of a dequantise warp (shared by the 1-CTA and 2-CTA kernels).
 // Warp dw handles row-block (dw & 7); of each lane's 16 packed bytes (two 32-wide k halves) a lane
@@ -181,8 +159,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(tfull_bar(b), 1);
             mbar_init(tempty_bar(b), kGemmEpilogueWarps);
         }
-        abort_flag[0] = 0;
-        abort_flag[1] = 0;
+        abort_flag[0] = 0;                                               // [0] abort, [1] abort of the exit drain,
+        abort_flag[1] = 0;                                               // [2], [3] "past griddepcontrol.wait" (see wait_expired)
+        abort_flag[2] = 0;
+        abort_flag[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), 2 * BN);
@@ -204,7 +184,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const uint8_t* wsrc = p.body + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
-                    QL_GTRACE(0, issued);
                     const int kc = it * CHUNKS;
                     const int nblk = min(CHUNKS, p.n_kc - kc);
                     const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
@@ -213,6 +192,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     if (!waited_dep) {                                   // x may come from the previous kernel
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         waited_dep = true;
+                        abort_flag[2] = 1;                               // from here on, waiting counts against the time limit
+                        abort_flag[3] = 1;
                     }
                     tma_load_2d(xs_addr(s), &x_map, it * kGemmKStep, m0, full_bar(s));
                     ++issued;
@@ -244,7 +225,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     // A tile written; the dequantise warps waited for the stage's TMA data, so x landed too
                     ok = mbar_wait(afull_bar(s), par, abort_flag, 0x300 + s);
                     if (!ok) break;
-                    QL_GTRACE(5, j * n_steps + it);
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
@@ -253,7 +233,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)         // +32 bytes along K inside the swizzle row
                         umma_f16_lo(tmem_d, a_lo + 2 * k4, b_lo + 2 * k4, idesc, 1u);
                     umma_commit(empty_bar(s));
-                    QL_GTRACE(6, j * n_steps + it);
                     if (++s == NS) { s = 0; par ^= 1; }
                 }
                 umma_commit(tfull_bar(buf));
@@ -273,11 +252,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
             for (int it = 0; it < n_steps; ++it, ++gstep) {
                 if (!mbar_wait(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
-                if (threadIdx.x == 64) QL_GTRACE(1, gstep);
                 dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(s));
                 fence_async_smem();                                      // generic-proxy writes -> visible to the MMA
                 __syncwarp();
-                if (threadIdx.x == 64) QL_GTRACE(3, gstep);
                 if (lane == 0) mbar_arrive(afull_bar(s));
                 if (++s == NS) { s = 0; par ^= 1; }
             }
@@ -325,6 +302,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 }
 
 // ----------------------------------------------------------------------------- host side
+// Tuning switches of the prefill kernels, read from the environment once per process (see library_config()).
+struct GemmConfig {
+    int force_bn = 0;        // QLINEAR_GEMM_BN: token-tile width of the single-CTA kernel (0 = choose per shape)
+    int force_split = 0;     // QLINEAR_GEMM_SPLIT: K parts of single-round layers in the CTA-pair kernel (0 = choose)
+    int force_tb = 0;        // QLINEAR_GEMM_TB: token blocks per tile of the CTA-pair kernel (0 = choose)
+    bool pair = true;        // QLINEAR_GEMM_PAIR=0 switches the CTA-pair kernel off
+};
+GemmConfig& gemm_config();
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -346,16 +332,38 @@ inline EncodeTiledFn get_encode_tiled()
     return fn;
 }
 
-inline ql_status gemm_plan(const Layout&, int, GemmPlan* p)
+// The tensor map of x depends only on (pointer, K, M, box rows); callers reuse a few activation buffers, so the
+// last encodings are kept (per process, a handful of entries) instead of calling the driver on every forward.
+inline bool x_tensor_map(const void* x, int K, int M, int box_rows, CUtensorMap* out)
 {
-    p->dummy = 0;
-    return QL_OK;
+    struct Entry { const void* x; int K, M, rows; CUtensorMap map; };
+    constexpr int kEntries = 16;
+    static Entry cache[kEntries] = {};
+    static int next = 0;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < kEntries; ++i)
+        if (cache[i].x == x && cache[i].K == K && cache[i].M == M && cache[i].rows == box_rows) { *out = cache[i].map; return true; }
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t gstr[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kGemmKStep, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    Entry e{x, K, M, box_rows, {}};
+    if (enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    cache[next] = e;
+    next = (next + 1) % kEntries;
+    *out = e.map;
+    return true;
 }
 
 inline int gemm_pick_bn(const Layout& L, int M, int num_sms)
 {
-    const char* f = std::getenv("QLINEAR_GEMM_BN");
-    if (f && *f) return std::atoi(f);
+    if (gemm_config().force_bn) return gemm_config().force_bn;
     if (M <= 32) return 32;
     if (M <= 64) return 64;
     if (M <= 128) return 128;
@@ -370,20 +378,11 @@ ql_status gemm_launch(const Layout& L, const uint8_t* blob, const void* x, void*
 {
     using S = GemmSmem<BITS, BN>;
     static_assert(S::kStages >= 2, "pipeline needs at least two stages");
-    EncodeTiledFn enc = get_encode_tiled();
-    if (!enc) return QL_ERR_CUDA;
     CUtensorMap map;
-    const cuuint64_t gdim[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
-    const cuuint64_t gstr[1] = {(cuuint64_t)L.K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kGemmKStep, (cuuint32_t)BN};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return QL_ERR_CUDA;
+    if (!x_tensor_map(x, L.K, M, BN, &map)) return QL_ERR_CUDA;
 
     auto kern = gemm_kernel<BITS, GROUPED, BN>;
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
             cudaGetLastError();
@@ -431,7 +430,7 @@ ql_status gemm_dispatch_bn(int bn, const Layout& L, const uint8_t* blob, const v
     return QL_ERR_INVALID_ARG;
 }
 
-inline ql_status gemm_forward(const Layout& L, const GemmPlan&, const uint8_t* blob, const void* x, void* y, int M,
+inline ql_status gemm_forward(const Layout& L, const uint8_t* blob, const void* x, void* y, int M,
                               cudaStream_t st, int device, bool pdl, int num_sms)
 {
     const int bn = gemm_pick_bn(L, M, num_sms);

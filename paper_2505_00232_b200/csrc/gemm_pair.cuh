@@ -6,8 +6,8 @@
 //
 // Roles per CTA are those of gemm.cuh.  Cross-CTA protocol (every CTA issues its own loads; nothing is loaded for a peer):
 //   * dequantise warps arrive on their own CTA's afull barrier (a warp dequantises only after its CTA's
-//     TMA data landed, so "A tile written" implies "x half landed"); in the peer CTA the otherwise idle
-//     MMA warp relays each completed afull phase to the leader with ONE remote arrive, on the leader's
+//     TMA data landed, so "A tile written" implies "x half landed"); in the peer CTA one spare warp per A
+//     slot relays each completed afull phase to the leader with ONE remote arrive, on the leader's
 //     afull barrier (17 arrivals there: its own 16 warps and the relay);
 //   * the leader's tcgen05.commit signals the empty / tfull barriers of BOTH CTAs (cluster mask 3 on the commit);
 //   * the epilogue warps of both CTAs arrive on the leader's tempty barrier (8 arrivals);
@@ -19,7 +19,7 @@ namespace ql {
 
 // Shared memory: a deep ring of TMA stages (this CTA's x half + packed weights) that covers the load
 // latency, and a short ring of dequantised A tiles (produced on chip, consumed a few hundred cycles later).
-// Warp roles: 0 producer, 1 MMA / relay, 2..22 except ids with (id % 4 == 1): 16 dequantise warps, 24..27 epilogue.
+// Warp roles: 0 producer, 1 MMA issuer, 2..22 except ids with (id % 4 == 1): 16 dequantise warps, 5/9/13/17/21: relays, 24..27 epilogue.
 constexpr int kPairFirstEpilogueWarp = 24;
 constexpr int kPairThreads = 28 * 32;
 
@@ -93,8 +93,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     auto full_bar = [&](int s) { return bar0 + 8 * s; };                 // local: this CTA's TMA data landed
     auto empty_bar = [&](int s) { return bar0 + 8 * (NS + s); };         // local, signalled by the leader's commit
     auto afull_bar = [&](int a) { return bar0 + 8 * (2 * NS + a); };     // local: this CTA's A tile written
-    auto aempty_bar = [&](int a) { return bar0 + 8 * (2 * NS + NA + a); };   // local, signalled by the leader's commit
-    auto pready_bar = [&](int a) { return bar0 + 8 * (2 * NS + 2 * NA + a); };   // leader: the peer's A slot is ready
     auto tfull_bar = [&](int b) { return bar0 + 8 * (2 * NS + 3 * NA + b); };        // local, signalled by the leader's commit
     auto tempty_bar = [&](int b) { return bar0 + 8 * (2 * NS + 3 * NA + 2 + b); };   // leader: both epilogues drained buffer b
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + S::kBarOffset + 8 * (2 * NS + 3 * NA + 4));
@@ -120,8 +118,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             mbar_init(tfull_bar(b), 1);
             mbar_init(tempty_bar(b), 2 * kGemmEpilogueWarps);
         }
-        abort_flag[0] = 0;
-        abort_flag[1] = 0;
+        abort_flag[0] = 0;                                               // [0] abort, [1] abort of the exit drain,
+        abort_flag[1] = 0;                                               // [2], [3] "past griddepcontrol.wait" (see wait_expired)
+        abort_flag[2] = 0;
+        abort_flag[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc_pair(smem_u32((const void*)tmem_slot), 2 * BN);
@@ -148,7 +148,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const uint8_t* wsrc = p.lbody[ly] + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
-                    QL_GTRACE(0, issued);
                     const int kc = (step0 + it) * CHUNKS;
                     const int nblk = min(CHUNKS, p.n_kc - kc);
                     const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
@@ -157,6 +156,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     if (!waited_dep) {
                         asm volatile("griddepcontrol.wait;" ::: "memory");
                         waited_dep = true;
+                        abort_flag[2] = 1;                               // from here on, waiting counts against the time limit
+                        abort_flag[3] = 1;
                     }
 #pragma unroll
                     for (int tb = 0; tb < TB; ++tb)
@@ -191,7 +192,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     // own A tile written (implies own x half landed) and the peer's likewise
                     // 16 local dequantise warps + the peer's relay lane: both A tiles written, both x halves landed
                     if (!mbar_wait(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
-                    QL_GTRACE(5, j * p.n_ksteps + it);
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
@@ -204,7 +204,6 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                             umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
                     }
                     umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
-                    QL_GTRACE(6, j * p.n_ksteps + it);
                     if (++s == NS) s = 0;
                     if (++a == NA) { a = 0; apar ^= 1; }
                 }
@@ -244,16 +243,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             const int n_steps = pair_unit(t, p).nsteps;
             for (int it = 0; it < n_steps; ++it, ++gstep) {
                 if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
-                if (threadIdx.x == 64) QL_GTRACE(1, gstep);
                 if (gstep >= NA) {
                     if (!mbar_wait(empty_bar(s_old), par_old, abort_flag, 0xB00 + s_old)) { ok = false; break; }
                     if (++s_old == NS) { s_old = 0; par_old ^= 1; }
                 }
-                if (threadIdx.x == 64) QL_GTRACE(2, gstep);
                 dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(a));
                 fence_async_smem();
                 __syncwarp();
-                if (threadIdx.x == 64) QL_GTRACE(3, gstep);
                 if (lane == 0) mbar_arrive(afull_bar(a));
                 if (++s == NS) { s = 0; par ^= 1; }
                 if (++a == NA) a = 0;
@@ -369,11 +365,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 inline int gemm_pair_split(int tiles /* of the last, partial round */, int n_ksteps, int num_sms, bool have_scratch)
 {
     if (!have_scratch) return 1;
-    const char* f = std::getenv("QLINEAR_GEMM_SPLIT");
     const int clusters = num_sms / 2;
     int split = 1;
     if (tiles == 0) return 1;
-    if (f && *f && std::atoi(f) > 0) split = std::atoi(f);
+    if (gemm_config().force_split > 0) split = gemm_config().force_split;
     else if (tiles * 4 <= clusters) split = 4;
     else if (tiles * 2 <= clusters) split = 2;
     while (split > 1 && (n_ksteps % split || n_ksteps / split < 8 || tiles * split > clusters)) split >>= 1;
@@ -381,8 +376,6 @@ inline int gemm_pair_split(int tiles /* of the last, partial round */, int n_kst
 }
 inline size_t gemm_pair_scratch_bytes(int num_sms) { return (size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float); }
 inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 8; }
-// A layer can only ever be split if it has few row-super-block pairs.
-inline bool gemm_pair_may_split(const Layout& L, int) { return (L.n_rsb % 2) == 0; }
 
 // The layers of one launch: all read the same x and agree in K and scheme; each has an even number of row
 // super-blocks.  L is the layout of the first one (K, chunking and scheme are taken from it).
@@ -400,19 +393,10 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
 {
     using S = GemmPairSmem<BITS, TB>;
     const Layout& L = *set.L[0];
-    EncodeTiledFn enc = get_encode_tiled();
-    if (!enc) return QL_ERR_CUDA;
     CUtensorMap map;
-    const cuuint64_t gdim[2] = {(cuuint64_t)L.K, (cuuint64_t)M};
-    const cuuint64_t gstr[1] = {(cuuint64_t)L.K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kGemmKStep, 128u};
-    const cuuint32_t estr[2] = {1, 1};
-    if (enc(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return QL_ERR_CUDA;
+    if (!x_tensor_map(x, L.K, M, 128, &map)) return QL_ERR_CUDA;
     auto kern = gemm_pair_kernel<BITS, GROUPED, TB>;
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
             cudaGetLastError();
@@ -473,9 +457,7 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
 // The pair kernel needs an even number of row super-blocks and enough tokens to fill a 256-wide tile.
 inline bool gemm_pair_applicable(const Layout& L, int M)
 {
-    const char* f = std::getenv("QLINEAR_GEMM_PAIR");
-    if (f && *f == '0') return false;
-    return (L.n_rsb % 2) == 0 && M > 128;
+    return gemm_config().pair && (L.n_rsb % 2) == 0 && M > 128;
 }
 
 inline ql_status gemm_pair_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st,
@@ -485,8 +467,7 @@ inline ql_status gemm_pair_forward(const GemmPairLayers& set, const void* x, int
     // bound by the tensor pipe and its operand traffic, not by dequantisation), so the wider tile only pays
     // where it saves rounds of the persistent grid.
     const Layout& L = *set.L[0];
-    const char* f = std::getenv("QLINEAR_GEMM_TB");
-    int tb = (f && *f) ? std::atoi(f) : 0;
+    int tb = gemm_config().force_tb;
     if (tb == 0) {
         const int clusters = num_sms / 2, pairs = set.n_rsb() / 2;
         const int tiles1 = pairs * ((M + 255) / 256), tiles2 = pairs * ((M + 511) / 512);

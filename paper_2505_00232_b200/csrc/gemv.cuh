@@ -52,14 +52,7 @@ struct GemvParams {
     int32_t x_bytes;                     // bytes of the x slab (the warp rings follow it)
 };
 
-__device__ __forceinline__ void mma_16816(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// Same instruction without `volatile`: the compiler may interleave independent MMA chains.
+// mma.m16n8k16 (fp16 in, fp32 accumulate), not `volatile`: the compiler may interleave independent MMA chains.
 __device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
 {
     asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"

@@ -32,20 +32,6 @@ constexpr int kStreamThreads = (kStreamConsumerWarps + 1) * 32;
 constexpr int kStreamMaxStages = 24;
 constexpr int kStreamPartialFloats = kStreamConsumerWarps * 128;        // one slot: 8 row-blocks x 16 rows x 8 tokens
 
-#ifdef QL_TRACE
-// Developer aid (not compiled by default): per-CTA %globaltimer stamps of the last 64 launches.
-constexpr int kTraceLaunches = 64, kTraceCtas = 600, kTracePoints = 8;
-__device__ unsigned long long g_trace[kTraceLaunches][kTraceCtas][kTracePoints];
-__device__ __forceinline__ unsigned long long trace_now()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#define QL_TRACE_AT(seq, pt) do { if ((int)blockIdx.x < kTraceCtas) g_trace[(seq) % kTraceLaunches][blockIdx.x][pt] = trace_now(); } while (0)
-#else
-#define QL_TRACE_AT(seq, pt) do { } while (0)
-#endif
 
 struct StreamParams {
     const uint8_t* body;
@@ -58,7 +44,6 @@ struct StreamParams {
     int32_t n_rsb, n_kc, block_bytes;
     int32_t P;                           // CTAs in the grid (<= number of blocks)
     int32_t stages;
-    int32_t trace_seq;                   // launch number (only read when built with QL_TRACE)
 };
 
 template <int BITS>
@@ -197,7 +182,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
     static_assert(NS % 2 == 0 && NS <= kStreamMaxStages, "the ring is consumed in stage pairs");
     extern __shared__ __align__(128) unsigned char smem_dyn[];
     __shared__ __align__(8) unsigned long long bars[2 * NS];
-    __shared__ uint32_t abort_word[2];
+    __shared__ uint32_t abort_word[3];           // [0] abort, [2] past griddepcontrol.wait (see wait_expired)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t B = (int64_t)p.n_rsb * p.n_kc;
@@ -211,13 +196,13 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
     auto empty_bar = [&](int s) { return bar0 + 8 * (NS + s); };
 
     if (threadIdx.x == 0) {
-        QL_TRACE_AT(p.trace_seq, 0);
         for (int s = 0; s < NS; ++s) {
             mbar_init(full_bar(s), 1);
             mbar_init(empty_bar(s), kStreamConsumerWarps);
         }
         abort_word[0] = 0;
         abort_word[1] = 0;
+        abort_word[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -242,9 +227,8 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
             // wait for the previous kernel, then add the x slices of those stages.
             const int pro = min(NS, nb);
             for (int i = 0; i < pro; ++i) issue_w(i, i);
-            QL_TRACE_AT(p.trace_seq, 1);
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            QL_TRACE_AT(p.trace_seq, 2);
+            abort_flag[2] = 1;
             int kcp = kc_first;
             for (int i = 0; i < pro; ++i) { issue_x(i, kcp); kcp = kcp + 1 == p.n_kc ? 0 : kcp + 1; }
             int s = 0;                                                   // pro == NS whenever this loop runs
@@ -291,7 +275,6 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
             if (j >= npairs) break;
             if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x700 + s)) return;
             if (!mbar_wait<true>(full_bar(s + 1), par, abort_flag, 0x700 + s + 1)) return;
-            if (j == 0 && threadIdx.x == 0) QL_TRACE_AT(p.trace_seq, 3);
             StreamFrag fa, fb;
             stream_load<BITS, GROUPED>(fa, smem_dyn + s * ST::kBytes, w_off, s_off, x_off);
             stream_load<BITS, GROUPED>(fb, smem_dyn + (s + 1) * ST::kBytes, w_off, s_off, x_off);
@@ -317,7 +300,6 @@ __global__ void __launch_bounds__(kStreamThreads, 3) gemv_stream_kernel(const St
         stream_math<BITS, GROUPED>(fa, total);
         advance(true);
     }
-    if (threadIdx.x == 0) QL_TRACE_AT(p.trace_seq, 5);
 }
 
 }  // namespace ql

@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -16,6 +17,9 @@
 namespace ql {
 // Set by a kernel that gave up a bounded wait: [0] = non-zero code identifying the wait, [1] = count.
 __device__ unsigned int g_device_flag[2];
+// Device-side alias of one word of pinned host memory (null until the first handle on the device exists): the
+// same code, readable by the host without synchronising.
+__device__ unsigned int* g_status_host;
 }  // namespace ql
 
 #include "dequant.cuh"
@@ -27,34 +31,7 @@ __device__ unsigned int g_device_flag[2];
 
 using namespace ql;
 
-struct GemvPlan {
-    int32_t ks_cta, cl, cps, x_stride, x_bytes, smem_bytes, grid;
-};
-
-struct qlinear_s {
-    Layout L;
-    const uint8_t* blob;
-    int device;
-    int num_sms;
-    int gemv_max_m;
-    bool pdl;
-    GemvPlan gemv[9];          // index = M (1..8)
-    GemvPlan group_gemv[9];    // the same for the last group of layers launched with this one in front
-    int group_rb;              // row-blocks of that group (0 = none yet)
-    GemmPlan gemm;
-    // streaming decode kernel
-    int gemv_kernel_choice;    // 0 = cluster kernel, 1 = streaming kernel
-    int stream_P, stream_stages;
-    float* stream_scratch;     // device, owned: [P][2][1024] fp32 partial sums
-    unsigned int* stream_counters;   // device, owned: [n_rsb][8], zero between launches
-    // prefill pair kernel, K-split of skinny layers
-    float* gemm_scratch;             // device, owned (nullptr if the layer can never be split)
-    unsigned int* gemm_counters;     // device, owned, zero between launches
-};
-
 namespace {
-
-constexpr int kGemvMaxSmem = 96 * 1024;
 
 int env_int(const char* name, int dflt)
 {
@@ -62,13 +39,104 @@ int env_int(const char* name, int dflt)
     return (v && *v) ? std::atoi(v) : dflt;
 }
 
+// Every QLINEAR_* switch, read from the environment ONCE per process (at the first call that needs one).
+struct Config {
+    int gemv_max_m;          // QLINEAR_GEMV_MAX_M: largest M served by the decode kernels (1..8)
+    bool pdl;                // QLINEAR_PDL: programmatic dependent launch attribute on every kernel
+    int warps_per_sm;        // QLINEAR_GEMV_WARPS_PER_SM: residency target of the cluster decode kernel
+    int force_ks;            // QLINEAR_GEMV_KS: forced K split of the cluster decode kernel (0 = planned)
+    bool xdirect;            // QLINEAR_GEMV_XDIRECT: x fragments straight from global memory
+    int kernel;              // QLINEAR_GEMV_KERNEL: 0 / 1 cluster kernel (default), 2 streaming kernel
+    int stream_ctas_per_sm, stream_stages;
+    GemmConfig gemm;
+    unsigned generation;     // bumped by qlinear_debug_reload_config (tests)
+};
+Config g_cfg;
+std::once_flag g_cfg_once;
+std::atomic<unsigned> g_getenv_reads{0};
+
+void load_config()
+{
+    Config c{};
+    c.gemv_max_m = std::max(1, std::min(8, env_int("QLINEAR_GEMV_MAX_M", 8)));
+    c.pdl = env_int("QLINEAR_PDL", 1) != 0;
+    c.warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
+    c.force_ks = env_int("QLINEAR_GEMV_KS", 0);
+    c.xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1) != 0;
+    const char* kc = std::getenv("QLINEAR_GEMV_KERNEL");
+    c.kernel = !kc ? 0 : !std::strcmp(kc, "cluster") ? 1 : !std::strcmp(kc, "stream") ? 2 : 0;
+    c.stream_ctas_per_sm = std::max(1, std::min(4, env_int("QLINEAR_STREAM_CTAS_PER_SM", 3)));
+    c.stream_stages = env_int("QLINEAR_STREAM_STAGES", kStreamMaxStages);
+    c.gemm.force_bn = env_int("QLINEAR_GEMM_BN", 0);
+    c.gemm.force_split = env_int("QLINEAR_GEMM_SPLIT", 0);
+    c.gemm.force_tb = env_int("QLINEAR_GEMM_TB", 0);
+    c.gemm.pair = env_int("QLINEAR_GEMM_PAIR", 1) != 0;
+    c.generation = g_cfg.generation + 1;
+    g_cfg = c;
+    g_getenv_reads.fetch_add(1);
+}
+const Config& config()
+{
+    std::call_once(g_cfg_once, load_config);
+    return g_cfg;
+}
+
+}  // namespace
+
+namespace ql {
+GemmConfig& gemm_config() { return const_cast<Config&>(config()).gemm; }
+}  // namespace ql
+
+namespace {
+
+struct GemvPlan {
+    int32_t ks_cta, cl, cps, x_stride, x_bytes, smem_bytes, grid;
+    double max_over_mean;    // chunks of the busiest SM over the mean, as the hardware would place the grid
+};
+
+// Device memory the library owns, ONE set per device, created with the first handle on that device and shared by
+// every handle there (kernels that use it run in stream order: see include/qlinear.h).
+struct DeviceState {
+    bool ready = false;
+    int sms = 0;
+    int handles = 0;
+    unsigned int* status_host = nullptr;     // pinned, mapped: the code of the last expired wait (0 = none)
+    float* gemm_scratch = nullptr;           // CTA-pair prefill kernel, K-split of single-round layers
+    unsigned int* gemm_counters = nullptr;
+    float* stream_scratch = nullptr;         // streaming decode kernel (only when QLINEAR_GEMV_KERNEL=stream)
+    unsigned int* stream_counters = nullptr;
+};
+constexpr int kMaxDevices = 64;
+constexpr int kStreamMaxRsb = 4096;          // row super-blocks the shared streaming-kernel counters cover
+DeviceState g_dev[kMaxDevices];
+std::mutex g_dev_mutex;
+
+}  // namespace
+
+struct qlinear_s {
+    // Immutable after qlinear_create.
+    Layout L;
+    const uint8_t* blob;
+    int device;
+    int num_sms;
+    int gemv_max_m;
+    bool pdl;
+    int n_rb;                  // row-blocks holding at least one real row
+    GemvPlan gemv[9];          // cluster decode kernel, index = M (1..8)
+    bool use_stream;
+    int stream_P, stream_stages;
+    DeviceState* dev;
+};
+
+namespace {
+
+constexpr int kGemvMaxSmem = 96 * 1024;
+
 // n_rb: row-blocks of the launch (one layer, or all layers of a group that shares x).
 GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
 {
-    const int warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
-    const int force_ks = env_int("QLINEAR_GEMV_KS", 0);
-    const int xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1);
-    const double target = (double)num_sms * warps_per_sm;
+    const Config& cfg = config();
+    const double target = (double)num_sms * cfg.warps_per_sm;
     GemvPlan best{};
     double best_score = -1e30;
     for (int ks_cta = 1; ks_cta <= 8; ks_cta *= 2)
@@ -80,7 +148,7 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
             const int x_stride = span + (((span * 2) % 128) == 0 ? 32 : 0);
             // x fragments straight from global memory need K to be a whole number of chunks (no bounds checks
             // in the kernel); otherwise x is staged in shared memory with zeros beyond K
-            const bool direct = xdirect && (L.K % L.chunk_k) == 0;
+            const bool direct = cfg.xdirect && (L.K % L.chunk_k) == 0;
             const int x_bytes = direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
@@ -90,11 +158,15 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
             // slices on half as many warps)
             double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 4 ? 1.25 : 0.0) - (cps < 2 ? 1.0 : 0.0);
             if (warps > target) score -= 2.0;                               // more CTAs than fit at once: a second wave
-            if (force_ks) score = (ks == force_ks) ? 0.0 : -1e29;
+            if (cfg.force_ks) score = (ks == cfg.force_ks) ? 0.0 : -1e29;
             if (score > best_score) {
                 best_score = score;
                 const int rb_per_cta = kGemvWarps / ks_cta;
-                best = GemvPlan{ks_cta, cl, cps, x_stride, x_bytes, smem, ((n_rb + rb_per_cta - 1) / rb_per_cta) * cl};
+                const int grid = ((n_rb + rb_per_cta - 1) / rb_per_cta) * cl;
+                // CTAs spread over the SMs one by one: the busiest SM holds ceil(grid / SMs) of them
+                const double per_sm = (double)grid / num_sms;
+                best = GemvPlan{ks_cta, cl, cps, x_stride, x_bytes, smem, grid,
+                                grid <= 4 * num_sms ? std::ceil(per_sm) / per_sm / eff : 2.0};
             }
         }
     return best;
@@ -127,16 +199,24 @@ cudaError_t launch(Kern kern, const Params& prm, dim3 grid, dim3 block, size_t s
     return cudaLaunchKernelEx(&cfg, kern, prm);
 }
 
+// cudaFuncSetAttribute once per (kernel instantiation, device); `flags` is that instantiation's table.
+template <typename Kern>
+cudaError_t ensure_smem_attr(Kern kern, std::atomic<bool>* flags, int device, int bytes)
+{
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (flags[device].load(std::memory_order_acquire)) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) flags[device].store(true, std::memory_order_release);
+    return e;
+}
+
 template <int BITS, bool GROUPED, bool XDIRECT>
 cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
 {
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[kMaxDevices];
     auto kern = gemv_kernel<BITS, GROUPED, XDIRECT>;
-    if (h->device >= 0 && h->device < 64 && !attr_set[h->device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvMaxSmem);
-        if (e != cudaSuccess) return e;
-        attr_set[h->device] = true;
-    }
+    cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, kGemvMaxSmem);
+    if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
 }
 
@@ -147,39 +227,35 @@ cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPla
                             : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
 }
 
-// One launch for n layers that read the same x (n == 1: the plain forward).
+// One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
+// call (integer arithmetic only); nothing is written to a handle.
 ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st)
 {
-    qlinear_s* h = hs[0];
+    const qlinear_s* h = hs[0];
     const Layout& L = h->L;
-    GemvParams prm{};
     int n_rb = 0;
+    for (int i = 0; i < n; ++i) n_rb += hs[i]->n_rb;
+    const GemvPlan pl = n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
+    cudaError_t e;
+    if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
+    GemvParams prm{};
+    int acc = 0;
     for (int i = 0; i < n; ++i) {
         const Layout& Li = hs[i]->L;
         prm.body[i] = hs[i]->blob + Li.body_offset;
         prm.chan_scales[i] = Li.grouped ? nullptr : reinterpret_cast<const __half*>(hs[i]->blob + Li.chan_scale_offset);
         prm.y[i] = static_cast<__half*>(ys[i]);
         prm.N[i] = Li.N;
-        n_rb += (Li.N + kRbRows - 1) / kRbRows;
-        prm.rb_end[i] = n_rb;
+        acc += hs[i]->n_rb;
+        prm.rb_end[i] = acc;
     }
     prm.n_layers = n;
-    GemvPlan pl;
-    if (n == 1) pl = h->gemv[M];
-    else {
-        if (h->group_rb != n_rb) {                                       // plans of the last group this layer led
-            for (int m = 1; m <= 8; ++m) h->group_gemv[m] = plan_gemv(L, n_rb, m, h->num_sms);
-            h->group_rb = n_rb;
-        }
-        pl = h->group_gemv[M];
-    }
     prm.x = static_cast<const __half*>(x);
     prm.M = M; prm.K = L.K;
     prm.n_rb = n_rb;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
-    cudaError_t e;
     if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st);
     else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st);
     else e = launch_gemv<4, false>(h, prm, pl, st);
@@ -189,13 +265,10 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
 template <int BITS, bool GROUPED, int NS>
 cudaError_t launch_stream_ns(const qlinear_s* h, const StreamParams& prm, cudaStream_t st)
 {
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[kMaxDevices];
     auto kern = gemv_stream_kernel<BITS, GROUPED, NS>;
-    if (h->device >= 0 && h->device < 64 && !attr_set[h->device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, NS * StreamStage<BITS>::kBytes);
-        if (e != cudaSuccess) return e;
-        attr_set[h->device] = true;
-    }
+    cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, NS * StreamStage<BITS>::kBytes);
+    if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(prm.P), dim3(kStreamThreads), (size_t)NS * StreamStage<BITS>::kBytes, st, 1, h->pdl);
 }
 
@@ -211,7 +284,7 @@ cudaError_t launch_stream(const qlinear_s* h, const StreamParams& prm, cudaStrea
     return cudaErrorInvalidValue;
 }
 
-ql_status forward_gemv_stream(qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
+ql_status forward_gemv_stream(const qlinear_s* h, const void* x, void* y, int M, cudaStream_t st)
 {
     const Layout& L = h->L;
     StreamParams prm{};
@@ -219,16 +292,12 @@ ql_status forward_gemv_stream(qlinear_s* h, const void* x, void* y, int M, cudaS
     prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
     prm.x = static_cast<const __half*>(x);
     prm.y = static_cast<__half*>(y);
-    prm.scratch = h->stream_scratch;
-    prm.counters = h->stream_counters;
+    prm.scratch = h->dev->stream_scratch;
+    prm.counters = h->dev->stream_counters;
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_rsb = L.n_rsb; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.P = h->stream_P;
     prm.stages = h->stream_stages;
-#ifdef QL_TRACE
-    static int trace_seq = 0;
-    prm.trace_seq = trace_seq++;
-#endif
     cudaError_t e;
     if (L.bits == 8) e = launch_stream<8, false>(h, prm, st);
     else if (L.grouped) e = launch_stream<4, true>(h, prm, st);
@@ -271,14 +340,16 @@ __global__ void __launch_bounds__(256) debug_unpack_kernel(const uint8_t* body, 
 __global__ void __launch_bounds__(32) expire_wait_kernel()
 {
     __shared__ __align__(8) unsigned long long bar;
-    __shared__ volatile uint32_t abort_word;
+    __shared__ volatile uint32_t abort_word[3];                          // [0] abort, [2] "dependency resolved"
     if (threadIdx.x == 0) {
-        abort_word = 0;
+        abort_word[0] = 0;
+        abort_word[1] = 0;
+        abort_word[2] = 1;
         mbar_init(smem_u32(&bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (threadIdx.x == 0) mbar_wait<true>(smem_u32(&bar), 0, &abort_word, 0x9A0);   // gives up, records the code
+    if (threadIdx.x == 0) mbar_wait<true>(smem_u32(&bar), 0, abort_word, 0x9A0);   // gives up, records the code
 }
 
 struct DeviceGuard {
@@ -295,6 +366,52 @@ struct DeviceGuard {
 
 }  // namespace
 
+namespace {
+
+// Creates the device's shared state on first use (the device must be current).  Called under g_dev_mutex.
+ql_status device_state_init(int device, int sms, DeviceState* d)
+{
+    if (d->ready) return QL_OK;
+    const Config& cfg = config();
+    d->sms = sms;
+    const size_t cb = gemm_pair_counter_count(sms) * sizeof(unsigned int);
+    bool ok = cudaHostAlloc(reinterpret_cast<void**>(&d->status_host), 64, cudaHostAllocMapped | cudaHostAllocPortable) == cudaSuccess;
+    unsigned int* status_dev = nullptr;
+    if (ok) {
+        d->status_host[0] = 0;
+        ok = cudaHostGetDevicePointer(reinterpret_cast<void**>(&status_dev), d->status_host, 0) == cudaSuccess &&
+             cudaMemcpyToSymbol(g_status_host, &status_dev, sizeof(status_dev)) == cudaSuccess;
+    }
+    ok = ok && cudaMalloc(&d->gemm_scratch, gemm_pair_scratch_bytes(sms)) == cudaSuccess &&
+         cudaMalloc(&d->gemm_counters, cb) == cudaSuccess && cudaMemset(d->gemm_counters, 0, cb) == cudaSuccess;
+    if (ok && cfg.kernel == 2) {
+        const size_t sbytes = (size_t)sms * 4 * 2 * kStreamPartialFloats * sizeof(float);
+        const size_t cbytes = (size_t)kStreamMaxRsb * 8 * sizeof(unsigned int);
+        ok = cudaMalloc(&d->stream_scratch, sbytes) == cudaSuccess && cudaMalloc(&d->stream_counters, cbytes) == cudaSuccess &&
+             cudaMemset(d->stream_counters, 0, cbytes) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        unsigned int* null_ptr = nullptr;
+        cudaMemcpyToSymbol(g_status_host, &null_ptr, sizeof(null_ptr));
+        cudaFreeHost(d->status_host); cudaFree(d->gemm_scratch); cudaFree(d->gemm_counters);
+        cudaFree(d->stream_scratch); cudaFree(d->stream_counters);
+        cudaGetLastError();
+        *d = DeviceState{};
+        return QL_ERR_CUDA;
+    }
+    d->ready = true;
+    return QL_OK;
+}
+
+// An earlier kernel on this device gave up a bounded wait: the host sees the code without synchronising.
+inline bool device_timed_out(const qlinear_s* h)
+{
+    return *reinterpret_cast<volatile unsigned int*>(h->dev->status_host) != 0;
+}
+
+}  // namespace
+
 extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_dev, int device, qlinear_t* out)
 {
     if (!d || !packed_dev || !out) return QL_ERR_INVALID_ARG;
@@ -304,53 +421,43 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
     if (reinterpret_cast<uintptr_t>(packed_dev) % 256) return QL_ERR_INVALID_ARG;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
-    if (device < 0 || device >= n_dev) return QL_ERR_INVALID_ARG;
+    if (device < 0 || device >= n_dev || device >= kMaxDevices) return QL_ERR_INVALID_ARG;
     int major = 0, sms = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
         return QL_ERR_CUDA;
     if (major != 10) return QL_ERR_ARCH;
+    const Config& cfg = config();
     qlinear_s* h = new (std::nothrow) qlinear_s();
     if (!h) return QL_ERR_ALLOC;
     h->L = L;
     h->blob = static_cast<const uint8_t*>(packed_dev);
     h->device = device;
     h->num_sms = sms;
-    h->gemv_max_m = std::max(1, std::min(8, env_int("QLINEAR_GEMV_MAX_M", 8)));
-    h->pdl = env_int("QLINEAR_PDL", 1) != 0;
-    for (int M = 1; M <= 8; ++M) h->gemv[M] = plan_gemv(L, (L.N + kRbRows - 1) / kRbRows, M, sms);
-    ql_status st = gemm_plan(L, sms, &h->gemm);
-    if (st != QL_OK) { delete h; return st; }
-    // streaming decode kernel: persistent grid, ring depth and per-handle scratch
+    h->gemv_max_m = cfg.gemv_max_m;
+    h->pdl = cfg.pdl;
+    h->n_rb = (L.N + kRbRows - 1) / kRbRows;
+    for (int M = 1; M <= 8; ++M) {
+        h->gemv[M] = plan_gemv(L, h->n_rb, M, sms);
+        if (h->gemv[M].grid <= 0 && M <= h->gemv_max_m) { delete h; return QL_ERR_UNSUPPORTED; }   // no decode plan fits this shape
+    }
     {
+        // streaming decode kernel (QLINEAR_GEMV_KERNEL=stream): persistent grid and ring depth
         const int stage_bytes = L.bits == 4 ? StreamStage<4>::kBytes : StreamStage<8>::kBytes;
-        const int ctas_per_sm = std::max(1, std::min(4, env_int("QLINEAR_STREAM_CTAS_PER_SM", 3)));
-        const int max_stages = std::min(env_int("QLINEAR_STREAM_STAGES", kStreamMaxStages), (220 * 1024 / ctas_per_sm - 1536) / stage_bytes);
+        const int max_stages = std::min(cfg.stream_stages, (220 * 1024 / cfg.stream_ctas_per_sm - 1536) / stage_bytes);
         h->stream_stages = max_stages >= 16 ? 16 : max_stages >= 12 ? 12 : max_stages >= 8 ? 8 : 6;   // instantiated ring depths
         const int64_t B = (int64_t)L.n_rsb * L.n_kc;
-        h->stream_P = (int)std::min<int64_t>(B, (int64_t)sms * ctas_per_sm);
-        const char* kc = std::getenv("QLINEAR_GEMV_KERNEL");
-        const int64_t body_bytes = B * L.block_bytes;
-        h->gemv_kernel_choice = (kc && !std::strcmp(kc, "cluster")) ? 0 : (kc && !std::strcmp(kc, "stream")) ? 1
-                                : (body_bytes >= (int64_t)env_int("QLINEAR_STREAM_MIN_MB", 1 << 20) * (1 << 20) ? 1 : 0);
-        if (L.bits == 4 && (L.K % 64)) h->gemv_kernel_choice = 0;       // the streaming kernel reads whole 64-k slices of x
+        h->stream_P = (int)std::min<int64_t>(B, (int64_t)sms * cfg.stream_ctas_per_sm);
+        // the streaming kernel reads whole 64-k slices of x and shares counters sized for kStreamMaxRsb row super-blocks
+        h->use_stream = cfg.kernel == 2 && !(L.bits == 4 && (L.K % 64)) && L.n_rsb <= kStreamMaxRsb;
+    }
+    {
         DeviceGuard guard(device);
-        const size_t sbytes = (size_t)h->stream_P * 2 * kStreamPartialFloats * sizeof(float);
-        const size_t cbytes = (size_t)L.n_rsb * 8 * sizeof(unsigned int);
-        if (!guard.ok || cudaMalloc(&h->stream_scratch, sbytes) != cudaSuccess) { cudaGetLastError(); delete h; return QL_ERR_CUDA; }
-        if (cudaMalloc(&h->stream_counters, cbytes) != cudaSuccess || cudaMemset(h->stream_counters, 0, cbytes) != cudaSuccess) {
-            cudaGetLastError(); cudaFree(h->stream_scratch); cudaFree(h->stream_counters); delete h; return QL_ERR_CUDA;
-        }
-        if (gemm_pair_may_split(L, sms)) {
-            const size_t cb = gemm_pair_counter_count(sms) * sizeof(unsigned int);
-            if (cudaMalloc(&h->gemm_scratch, gemm_pair_scratch_bytes(sms)) != cudaSuccess ||
-                cudaMalloc(&h->gemm_counters, cb) != cudaSuccess || cudaMemset(h->gemm_counters, 0, cb) != cudaSuccess) {
-                cudaGetLastError();
-                cudaFree(h->stream_scratch); cudaFree(h->stream_counters); cudaFree(h->gemm_scratch); cudaFree(h->gemm_counters);
-                delete h;
-                return QL_ERR_CUDA;
-            }
-        }
+        std::lock_guard<std::mutex> lock(g_dev_mutex);
+        ql_status st = guard.ok ? device_state_init(device, sms, &g_dev[device]) : QL_ERR_CUDA;
+        if (st != QL_OK) { cudaGetLastError(); delete h; return st; }
+        h->dev = &g_dev[device];
+        ++h->dev->handles;
     }
     *out = h;
     return QL_OK;
@@ -367,16 +474,17 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!h || !x || !y || M < 1) return QL_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
     if ((int64_t)M * h->L.K > INT32_MAX || (int64_t)M * h->L.N > INT32_MAX) return QL_ERR_INVALID_ARG;
+    if (device_timed_out(h)) return QL_ERR_DEVICE_TIMEOUT;
     DeviceGuard guard(h->device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (M <= h->gemv_max_m) return h->gemv_kernel_choice ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
+    if (M <= h->gemv_max_m) return h->use_stream ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
     if (gemm_pair_applicable(h->L, M)) {
         GemmPairLayers set{};
         set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y;
-        return gemm_pair_forward(set, x, M, st, h->device, h->pdl, h->num_sms, h->gemm_scratch, h->gemm_counters);
+        return gemm_pair_forward(set, x, M, st, h->device, h->pdl, h->num_sms, h->dev->gemm_scratch, h->dev->gemm_counters);
     }
-    return gemm_forward(h->L, h->gemm, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
+    return gemm_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
 
 extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x, void* const* ys, int32_t M, void* stream)
@@ -389,8 +497,9 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         if ((int64_t)M * b.N > INT32_MAX) return QL_ERR_INVALID_ARG;
     }
     if ((reinterpret_cast<uintptr_t>(x) & 15) || (int64_t)M * hs[0]->L.K > INT32_MAX) return QL_ERR_INVALID_ARG;
+    if (device_timed_out(hs[0])) return QL_ERR_DEVICE_TIMEOUT;
     // One kernel where the decode kernel serves the call; otherwise the layers run one after the other.
-    if (n > 1 && M <= hs[0]->gemv_max_m && hs[0]->gemv_kernel_choice == 0) {
+    if (n > 1 && M <= hs[0]->gemv_max_m && !hs[0]->use_stream) {
         DeviceGuard guard(hs[0]->device);
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
         return forward_gemv(const_cast<qlinear_s* const*>(hs), n, x, ys, M, static_cast<cudaStream_t>(stream));
@@ -405,7 +514,7 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
             set.n = n;
             for (int i = 0; i < n; ++i) { set.L[i] = &hs[i]->L; set.blob[i] = hs[i]->blob; set.y[i] = ys[i]; }
             return gemm_pair_forward(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
-                                     hs[0]->gemm_scratch, hs[0]->gemm_counters);
+                                     hs[0]->dev->gemm_scratch, hs[0]->dev->gemm_counters);
         }
     }
     for (int i = 0; i < n; ++i) {
@@ -505,14 +614,11 @@ ql_status static_setup(int device, StaticDevice** out)
 template <int BITS, bool GROUPED>
 cudaError_t launch_stream_static(const StreamParams& prm, cudaStream_t st, int device)
 {
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[kMaxDevices];
     auto kern = gemv_stream_kernel<BITS, GROUPED, kStaticStages>;
     const size_t smem = (size_t)kStaticStages * StreamStage<BITS>::kBytes;
-    if (!attr_set[device]) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        attr_set[device] = true;
-    }
+    cudaError_t e = ensure_smem_attr(kern, attr_set, device, (int)smem);
+    if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(prm.P), dim3(kStreamThreads), smem, st, 1, false);
 }
 
@@ -529,6 +635,12 @@ extern "C" ql_status qlinear_decode_static(const qlinear_desc* d, const void* pa
     if (!make_layout(d->N, d->K, d->bits, d->group, &L)) return QL_ERR_UNSUPPORTED;
     if (L.n_rsb > kStaticMaxRsb) return QL_ERR_UNSUPPORTED;              // beyond the static counters
     if (L.bits == 4 && (L.K % 64)) return QL_ERR_UNSUPPORTED;            // the streaming kernel reads whole 64-k slices
+    if (device < 0 || device >= kMaxDevices) return QL_ERR_INVALID_ARG;
+    {
+        int n_dev = 0;
+        if (cudaGetDeviceCount(&n_dev) != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
+        if (device >= n_dev) return QL_ERR_INVALID_ARG;
+    }
     DeviceGuard guard(device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     StaticDevice* dev = nullptr;
@@ -582,8 +694,13 @@ extern "C" ql_status qlinear_device_status(qlinear_t h, uint32_t* detail)
     if (cudaMemcpyFromSymbol(flag, g_device_flag, sizeof(flag)) != cudaSuccess) { cudaGetLastError(); return QL_ERR_CUDA; }
     if (detail) *detail = flag[0];
     if (flag[0] == 0) return QL_OK;
+    // Clear the condition, and with it whatever an abandoned launch left in the shared arrival counters.
     const unsigned int zero[2] = {0, 0};
     cudaMemcpyToSymbol(g_device_flag, zero, sizeof(zero));
+    h->dev->status_host[0] = 0;
+    cudaMemset(h->dev->gemm_counters, 0, gemm_pair_counter_count(h->dev->sms) * sizeof(unsigned int));
+    if (h->dev->stream_counters) cudaMemset(h->dev->stream_counters, 0, (size_t)kStreamMaxRsb * 8 * sizeof(unsigned int));
+    cudaDeviceSynchronize();
     return QL_ERR_DEVICE_TIMEOUT;
 }
 
@@ -591,15 +708,24 @@ extern "C" ql_status qlinear_destroy(qlinear_t h)
 {
     if (!h) return QL_OK;
     {
-        DeviceGuard guard(h->device);
-        cudaFree(h->stream_scratch);
-        cudaFree(h->stream_counters);
-        cudaFree(h->gemm_scratch);
-        cudaFree(h->gemm_counters);
+        std::lock_guard<std::mutex> lock(g_dev_mutex);
+        --h->dev->handles;                   // the device's shared state stays for the next handle (a few tens of MB)
     }
     delete h;
     return QL_OK;
 }
+
+extern "C" int32_t qlinear_debug_plan(qlinear_t h, int32_t M, int32_t* out, int32_t n_out)
+{
+    if (!h || M < 1 || M > 8 || !out) return 0;
+    const int32_t v[8] = {h->use_stream ? 3 : 1, h->gemv[M].grid, h->gemv[M].cl, h->gemv[M].ks_cta, h->gemv[M].cps,
+                          (int32_t)(1000 * h->gemv[M].max_over_mean), h->n_rb, h->L.n_kc};
+    int n = n_out < 8 ? n_out : 8;
+    for (int i = 0; i < n; ++i) out[i] = v[i];
+    return n;
+}
+
+extern "C" uint32_t qlinear_debug_config_reads(void) { config(); return g_getenv_reads.load(); }
 
 extern "C" const char* qlinear_status_string(ql_status s)
 {
@@ -615,15 +741,5 @@ extern "C" const char* qlinear_status_string(ql_status s)
     return "unknown status";
 }
 
-#ifdef QL_TRACE
-extern "C" int qlinear_debug_read_gemm_trace(unsigned long long* out, size_t bytes)
-{
-    return (int)cudaMemcpyFromSymbol(out, g_gemm_trace, bytes < sizeof(g_gemm_trace) ? bytes : sizeof(g_gemm_trace));
-}
-extern "C" int qlinear_debug_read_trace(unsigned long long* out, size_t bytes)
-{
-    return (int)cudaMemcpyFromSymbol(out, g_trace, bytes < sizeof(g_trace) ? bytes : sizeof(g_trace));
-}
-#endif
 
 extern "C" uint32_t qlinear_version(void) { return (1u << 16) | 0u; }

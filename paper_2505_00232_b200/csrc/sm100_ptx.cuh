@@ -12,6 +12,27 @@ constexpr uint32_t kSuspendHintNs = 20000;     // a waiting thread is suspended 
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// A wait gave up: record the code for this CTA, for the device (g_device_flag) and, without waiting for any
+// synchronisation, for the host (g_status_host points to pinned host memory mapped into the device, or is null).
+__device__ __forceinline__ void report_timeout(volatile uint32_t* abort_flag, uint32_t code)
+{
+    *abort_flag = code;
+    atomicExch(&g_device_flag[0], code);
+    atomicAdd(&g_device_flag[1], 1u);
+    if (g_status_host) {
+        *reinterpret_cast<volatile unsigned int*>(g_status_host) = code;
+        __threadfence_system();
+    }
+}
+// abort_flag[2] is the CTA's "dependency resolved" word: a thread sets it once it is past griddepcontrol.wait.
+// While it is zero the kernel this one depends on is still running, and time spent waiting does not count.
+__device__ __forceinline__ bool wait_expired(long long& t0, volatile uint32_t* abort_flag)
+{
+    if (clock64() - t0 <= kWaitCycles) return false;
+    if (abort_flag[2] == 0) { t0 = clock64(); return false; }
+    return true;
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
@@ -34,34 +55,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Same test without a suspend hint: returns at once, for a hot poll by a thread on the critical path.
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded hot wait (polls, never suspended): lowest wake-up latency, costs issue slots while waiting.
-__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code)
-{
-    if (mbar_test_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_test_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = code;
-            atomicExch(&g_device_flag[0], code);
-            atomicAdd(&g_device_flag[1], 1u);
-            return false;
-        }
-    }
-}
-
 // Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.
 // SLEEP: back off between polls (for waits that are long and off the critical path, so that the issue
 // slots go to warps that have work); without it the wait wakes up as soon as the phase completes.
@@ -69,17 +62,15 @@ template <bool SLEEP = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 32; ++i) {
             if (mbar_try_wait(bar, parity)) return true;
             if (SLEEP) __nanosleep(64);
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = code;
-            atomicExch(&g_device_flag[0], code);
-            atomicAdd(&g_device_flag[1], 1u);
+        if (wait_expired(t0, abort_flag)) {
+            report_timeout(abort_flag, code);
             return false;
         }
     }
@@ -110,31 +101,12 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
 
-// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);          // start address
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset
-    d |= (uint64_t)1 << 46;                           // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                           // SWIZZLE_128B
-    return d;
-}
-
 // Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128, N = n.
 __host__ __device__ constexpr uint32_t umma_idesc_f16(int n)
 {
     return (1u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "setp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
 // Lean issue forms for the MMA loop: the descriptors are passed as 32-bit halves (the high half is a
 // constant of the layout, the low half is the start address field), so that the single issuing thread
 // spends two integer adds per MMA instead of rebuilding 64-bit descriptors.
@@ -194,33 +166,6 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t cta)
                  "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
                  ::"r"(bar), "r"(cta) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-                 "selp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait on a barrier that CTAs of the whole cluster arrive on.
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code)
-{
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        for (int i = 0; i < 32; ++i)
-            if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *abort_flag = code;
-            atomicExch(&g_device_flag[0], code);
-            atomicAdd(&g_device_flag[1], 1u);
-            return false;
-        }
-    }
-}
-
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols)
 {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -229,14 +174,6 @@ __device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncol
 __device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols)
 {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-// One MMA across a CTA pair: D (256 x N, 128 rows per CTA) += A (each CTA's own 128 rows) x B (N/2 rows per CTA).
-__device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n\t.reg .pred p;\n\t"
-                 "setp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 // Arrive, when all MMAs issued so far have retired, on the mbarrier at this offset in both CTAs of the pair.
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar)

@@ -138,3 +138,16 @@ def test_host_calls_that_need_no_device(P):
     assert P.lib.qlinear_forward_group(hs, 0, ctypes.c_void_p(16), ys, 1, None) == 1
     assert P.lib.qlinear_forward_group(hs, 5, ctypes.c_void_p(16), ys, 1, None) == 1
     assert P.lib.qlinear_forward_group(hs, 2, ctypes.c_void_p(16), ys, 1, None) == 1      # null handles
+
+
+def test_environment_is_read_once(P, monkeypatch):
+    """Every QLINEAR_* switch is read at the first call that needs one, and never again."""
+    n = P.lib.qlinear_debug_config_reads()
+    assert n == 1
+    monkeypatch.setenv("QLINEAR_GEMV_MAX_M", "2")
+    monkeypatch.setenv("QLINEAR_GEMM_PAIR", "0")
+    assert P.lib.qlinear_debug_config_reads() == 1
+    h = ctypes.c_void_p()
+    d = P.Desc(16, 64, 8, 0).c()
+    P.lib.qlinear_create(ctypes.byref(d), ctypes.c_void_p(256), 0, ctypes.byref(h))   # fails without a device; reads nothing new
+    assert P.lib.qlinear_debug_config_reads() == 1
