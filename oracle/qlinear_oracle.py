@@ -22,7 +22,10 @@ the three loops out with ascending k; the tests require the two to agree.
 
 Parity pins: tests/test_oracle_pins.py (worked examples stored under
 tests/golden/, brute force over all byte values, one-hot / zero / closed-form
-cases, power-of-two and negation invariants, a double-rounding trap).
+cases, power-of-two and negation invariants, a double-rounding trap) and
+tests/test_oracle_pins_next.py for the three extensions further down (fused
+gating, Section 3.6; int8 activation quantisation, Section 3.7; the KV cache as
+weights, Section 3.8).  No function here is unpinned.
 """
 from __future__ import annotations
 
@@ -101,6 +104,122 @@ def check_against(y_test: np.ndarray, y64: np.ndarray, A: np.ndarray):
         ratio = np.where(A > 0, np.abs(d) / A, np.where(d == 0, 0.0, np.inf))
     worst = float(ratio.max(initial=0.0))
     return (rel <= REL_L2_TOL and worst <= ELEM_TOL), rel, worst
+
+
+# ----------------------------------------------------------------------------- fused gating (paper Section 3.6)
+# The paper's operator fusion merges "element-wise operators from two branches with a fully connected
+# operator" (Section 3.6, the left example of its fusion figure): in the feed-forward block the gate and up
+# projections read the same x and meet in an element-wise product, y = act(W_gate x) * (W_up x).  The paper
+# names no activation; the model families it evaluates use SiLU (Llama) and the tanh form of GELU (Gemma).
+# Reading: both projections stay unrounded until the product (the fused kernel keeps them in fp32
+# accumulators), and the product is rounded to fp16 once.
+_SQRT_2_OVER_PI = 0.7978845608028654  # sqrt(2 / pi)
+
+
+def activation(g: np.ndarray, act: str) -> np.ndarray:
+    """fp64 activation by its textbook formula: 'identity', 'silu' (g * sigmoid(g)), 'gelu_tanh'."""
+    g = np.asarray(g, dtype=np.float64)
+    if act == "identity":
+        return g.copy()
+    if act == "silu":
+        return g / (1.0 + np.exp(-g))
+    if act == "gelu_tanh":
+        return 0.5 * g * (1.0 + np.tanh(_SQRT_2_OVER_PI * (g + 0.044715 * g * g * g)))
+    raise ValueError(act)
+
+
+# Largest slope of the activation (bounds how an error in the gate projection reaches the product).
+ACT_LIPSCHITZ = {"identity": 1.0, "silu": 1.0999, "gelu_tanh": 1.1290}
+
+
+def gated_linear(x, q_gate, s_gate, q_up, s_up, group: int, act: str):
+    """(y64, bound, y16): y64 = act(gate64) * up64 with gate64 / up64 the two `linear` results.
+    bound[m,n] is the per-element acceptance bound that follows from the linear layer's own
+    (|d gate| <= ELEM_TOL * A_gate, |d up| <= ELEM_TOL * A_up), first order, plus one fp16 rounding:
+        ELEM_TOL * (L_act * |up64| * A_gate + |act(gate64)| * A_up) + 2^-10 * |y64|."""
+    g64, A_g, _ = linear(x, q_gate, s_gate, group)
+    u64, A_u, _ = linear(x, q_up, s_up, group)
+    a = activation(g64, act)
+    y64 = a * u64
+    bound = ELEM_TOL * (ACT_LIPSCHITZ[act] * np.abs(u64) * A_g + np.abs(a) * A_u) + 2.0 ** -10 * np.abs(y64)
+    with np.errstate(over="ignore"):
+        y16 = y64.astype(np.float16)
+    return y64, bound, y16
+
+
+def check_gated(y_test, y64, bound):
+    """Returns (ok, rel_l2, worst |y - y64| / bound): rel-L2 <= REL_L2_TOL over the whole output, every element inside its bound."""
+    d = np.asarray(y_test).astype(np.float64) - y64
+    den = np.linalg.norm(y64)
+    rel = float(np.linalg.norm(d) / den) if den > 0 else float(np.linalg.norm(d))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ratio = np.where(bound > 0, np.abs(d) / bound, np.where(d == 0, 0.0, np.inf))
+    worst = float(ratio.max(initial=0.0))
+    return (rel <= REL_L2_TOL and worst <= 1.0), rel, worst
+
+
+# ----------------------------------------------------------------------------- activation quantisation (paper Section 3.7)
+# The method the paper describes for operators with external weights quantises the ACTIVATIONS too: a
+# quantisation kernel "converts the floating-point input activations to 8-bit integers and computes the
+# requisite quantization parameters", a second kernel multiplies them with the pre-quantised weights using
+# integer instructions and "perform[s] dequantization on the output activations" (prefill); in decode the
+# quantisation happens inside the fully-connected kernel.  The steps below follow that order.  The paper
+# gives neither the granularity nor the rounding; the readings taken (recorded in the design notes):
+#   * one scale per token (row of x), symmetric, zero-point 0:  scale_x[m] = amax_m / 127,  amax_m = max_k |x[m,k]|
+#   * a floating-point value decides an integer here, so the decision is taken in ONE stated precision, fp32,
+#     with these IEEE operations:  r = 127 / amax (division),  v = x * r (multiplication),
+#     xq = round-half-to-even(v) clamped to [-127, 127];  a row of zeros gets scale 1 and xq = 0
+#   * the integer dot products are exact (accumulated in int64 here), one per scale group of the weights
+#   * output dequantisation  y = scale_x[m] * sum_g s[n,g] * acc[m,n,g],  in fp64 here from the fp32 scale_x
+#     and the fp16 weight scales, then one rounding to fp16.
+
+
+def quantize_activations(x: np.ndarray):
+    """x fp16 [M, K] -> (xq int8 [M, K], scale_x float32 [M]) by the fp32 steps stated above."""
+    x32 = np.asarray(x, dtype=np.float16).astype(np.float32)
+    amax = np.abs(x32).max(axis=1)
+    live = amax > 0
+    safe = np.where(live, amax, np.float32(1.0)).astype(np.float32)
+    r = (np.float32(127.0) / safe).astype(np.float32)                    # one IEEE fp32 division per token
+    v = (x32 * r[:, None]).astype(np.float32)                            # one IEEE fp32 multiplication per element
+    xq = np.clip(np.rint(v), -127, 127).astype(np.int8)                  # rint = round half to even
+    scale = np.where(live, (safe / np.float32(127.0)).astype(np.float32), np.float32(1.0)).astype(np.float32)
+    return xq, scale
+
+
+def linear_int8_activations(x, q, s, group: int):
+    """(y64, acc, xq, scale_x, y16): the linear layer with per-token int8 activations.
+    acc int64 [M, N, K/G] are the exact integer dot products per scale group."""
+    q = np.asarray(q, dtype=np.int8)
+    N, K = q.shape
+    G = K if group == 0 else group
+    xq, scale_x = quantize_activations(x)
+    M = xq.shape[0]
+    acc = np.einsum("mgk,ngk->mng", xq.astype(np.int64).reshape(M, K // G, G), q.astype(np.int64).reshape(N, K // G, G))
+    s64 = np.asarray(s, dtype=np.float16).reshape(N, K // G).astype(np.float64)
+    y64 = scale_x.astype(np.float64)[:, None] * np.einsum("mng,ng->mn", acc.astype(np.float64), s64)
+    with np.errstate(over="ignore"):
+        y16 = y64.astype(np.float16)
+    return y64, acc, xq, scale_x, y16
+
+
+# ----------------------------------------------------------------------------- KV cache as weights (paper Section 3.8)
+# The attention matmuls are run as operators with weights: the K cache is stored O x I with O = cache
+# positions and I = head dimension (it "represent[s] K^T for the QK^T computation"), the V cache O x I with
+# O = head dimension and I = cache positions, so that the second product comes out as [query rows, d_h].
+# Both are then the linear layer above; only the meaning of the axes differs.  The caches are held in the
+# int8 per-output-channel format of Section 4.2 (one scale per cached key for K; one scale per head
+# dimension for V), the reading recorded in the design notes: the paper does not say how its cache is stored.
+
+
+def kv_scores(qry, k_q, k_s):
+    """scores64 [R, T] = qry [R, d_h] . Kcache^T, K cache k_q int8 [T, d_h] (O = T, I = d_h), k_s fp16 [T]."""
+    return linear(qry, k_q, k_s, 0)
+
+
+def kv_output(prob, v_q, v_s):
+    """out64 [R, d_h] = prob [R, T] . V, V cache v_q int8 [d_h, T] (O = d_h, I = T), v_s fp16 [d_h]."""
+    return linear(prob, v_q, v_s, 0)
 
 
 # ----------------------------------------------------------------------------- C oracle

@@ -1,0 +1,186 @@
+"""Pins of the oracle's three extensions: fused gating (paper Section 3.6), int8 activation quantisation
+(Section 3.7) and the KV cache held as weights (Section 3.8).  CPU only.  Each pin checks the oracle against
+something other than itself: hand-computed examples (tests/golden), closed forms and identities of the
+activations, a library routine, brute force in plain Python integers, or the special case in which the
+extension must fall back onto the plain linear layer."""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import qlinear_oracle as O
+from workloads import configs as C
+
+
+def rand_layer(seed, N, K, bits, group):
+    layer = C.LayerSpec("t", N, K, bits, group, *((-8, 7) if bits == 4 else (-128, 127)))
+    return C.layer_weights(seed, layer)
+
+
+# ----------------------------------------------------------------------------- fused gating
+def test_example_F_gated_silu(golden):
+    e = golden["F_gated_silu"]
+    x = np.array(e["x"], np.float16)
+    y64, bound, y16 = O.gated_linear(x, np.array(e["q_gate"], np.int8), np.array(e["s_gate"], np.float16),
+                                     np.array(e["q_up"], np.int8), np.array(e["s_up"], np.float16), e["group"], "silu")
+    np.testing.assert_allclose(y64, np.array(e["y64"]), rtol=1e-15, atol=0)
+    assert (bound > 0).all()
+    assert (y16 == y64.astype(np.float16)).all()
+
+
+@pytest.mark.parametrize("act", ["silu", "gelu_tanh"])
+def test_activation_identities_and_closed_values(act):
+    g = np.linspace(-12, 12, 4801)
+    a = O.activation(g, act)
+    np.testing.assert_allclose(a - O.activation(-g, act), g, rtol=0, atol=1e-14)     # act(g) - act(-g) = g for both
+    assert O.activation(np.array([0.0]), act)[0] == 0.0
+    assert abs(O.activation(np.array([30.0]), act)[0] - 30.0) < 1e-10               # identity far to the right
+    assert abs(O.activation(np.array([-30.0]), act)[0]) < 1e-10                     # zero far to the left
+    if act == "silu":
+        assert abs(O.activation(np.array([math.log(3.0)]), act)[0] - 0.75 * math.log(3.0)) < 1e-15   # sigmoid(ln 3) = 3/4
+    # the slope bound used in the acceptance bound is the true maximum slope, to three digits
+    slope = np.abs(np.diff(O.activation(np.linspace(-8, 8, 1_600_001), act)) / 1e-5)
+    assert O.ACT_LIPSCHITZ[act] - 2e-3 < slope.max() <= O.ACT_LIPSCHITZ[act]
+
+
+def test_activations_agree_with_library_routines():
+    torch = pytest.importorskip("torch")
+    g = np.linspace(-9, 9, 2001)
+    t = torch.from_numpy(g)
+    np.testing.assert_allclose(O.activation(g, "silu"), torch.nn.functional.silu(t).numpy(), rtol=1e-14, atol=1e-16)
+    np.testing.assert_allclose(O.activation(g, "gelu_tanh"), torch.nn.functional.gelu(t, approximate="tanh").numpy(), rtol=1e-13, atol=2e-15)   # 1 + tanh cancels far to the left
+
+
+@pytest.mark.parametrize("bits,group", [(8, 0), (4, 32), (4, 0)])
+def test_gated_identity_is_the_product_of_two_linear_calls_and_branches_are_not_swapped(bits, group):
+    qg, sg = rand_layer(11, 24, 128, bits, group)
+    qu, su = rand_layer(12, 24, 128, bits, group)
+    x = C.layer_activations(13, C.LayerSpec("t", 24, 128, bits, group, 0, 0), 3)
+    g64, _, _ = O.linear(x, qg, sg, group)
+    u64, _, _ = O.linear(x, qu, su, group)
+    y64, _, _ = O.gated_linear(x, qg, sg, qu, su, group, "identity")
+    assert (y64 == g64 * u64).all()
+    ys, _, _ = O.gated_linear(x, qg, sg, qu, su, group, "silu")
+    yt, _, _ = O.gated_linear(x, qu, su, qg, sg, group, "silu")                   # branches swapped: a different function
+    np.testing.assert_allclose(ys, g64 / (1 + np.exp(-g64)) * u64, rtol=1e-15)
+    np.testing.assert_allclose(yt, u64 / (1 + np.exp(-u64)) * g64, rtol=1e-15)
+    assert np.abs(ys - yt).max() > 1e-3
+
+
+def test_gated_bound_holds_for_an_fp32_emulation_of_the_fused_kernel():
+    """fp16-rounded grouped weights, fp32 accumulation of both branches, fp32 activation, one fp16 rounding."""
+    K, N, M = 4096, 48, 4
+    qg, sg = rand_layer(21, N, K, 4, 32)
+    qu, su = rand_layer(22, N, K, 4, 32)
+    x = C.layer_activations(23, C.LayerSpec("t", N, K, 4, 32, 0, 0), M)
+    def branch32(q, s):
+        w16 = (np.repeat(s.astype(np.float32), 32, axis=1) * q.astype(np.float32)).astype(np.float16).astype(np.float32)
+        acc = np.zeros((M, N), np.float32)
+        for k0 in range(0, K, 64):
+            acc = (acc + x[:, k0:k0 + 64].astype(np.float32) @ w16[:, k0:k0 + 64].T).astype(np.float32)
+        return acc
+    g32, u32 = branch32(qg, sg), branch32(qu, su)
+    y = ((g32 / (np.float32(1) + np.exp(-g32))) * u32).astype(np.float16)
+    y64, bound, _ = O.gated_linear(x, qg, sg, qu, su, 32, "silu")
+    ok, rel, worst = O.check_gated(y, y64, bound)
+    assert ok and rel < 6e-4 and worst < 0.5, (rel, worst)
+    bad = y.copy()
+    bad[1, 5] = np.float16(float(bad[1, 5]) + 3 * float(bound[1, 5]) + 1e-3)
+    assert not O.check_gated(bad, y64, bound)[0]
+
+
+# ----------------------------------------------------------------------------- activation quantisation
+def test_example_G_activation_quantisation(golden):
+    e = golden["G_act_quant"]
+    x = np.array(e["x"], np.float16)
+    xq, sx = O.quantize_activations(x)
+    assert xq.tolist() == e["xq"] and sx.tolist() == e["scale_x"]
+    y64, acc, _, _, _ = O.linear_int8_activations(x, np.array(e["q"], np.int8), np.array(e["s"], np.float16), 0)
+    assert acc.tolist() == e["acc"] and y64.tolist() == e["y64"]
+
+
+def test_quantisation_rounds_half_to_even_clamps_and_handles_zero_rows():
+    # amax = 127 * 2^-3 makes r = 8 exactly: x * 8 is exact, ties are real ties
+    x = np.array([[127 / 8, 0.5 / 8, 1.5 / 8, 2.5 / 8, -0.5 / 8, -1.5 / 8, -126.5 / 8, 63.5 / 8],
+                  [0, 0, 0, 0, 0, 0, 0, 0],
+                  [-3.0, 1.0, 0.0, 3.0, 2.9, -2.9, 0.01, -0.01]], np.float16)
+    assert all(float(v) * 8 == round(float(v) * 8 * 2) / 2 for v in x[0])           # the fixture is exact in fp16
+    xq, sx = O.quantize_activations(x)
+    assert xq[0].tolist() == [127, 0, 2, 2, 0, -2, -126, 64]
+    assert sx[0] == np.float32(1 / 8) and sx[1] == np.float32(1.0) and not xq[1].any()
+    assert xq[2, 0] == -127 and xq[2, 3] == 127 and np.abs(xq).max() == 127         # the largest magnitude maps to +-127
+    # reconstruction error is at most half a step (plus fp32 round-off of the two operations)
+    err = np.abs(x.astype(np.float64) - sx.astype(np.float64)[:, None] * xq)
+    assert (err <= 0.5 * sx.astype(np.float64)[:, None] * (1 + 1e-6)).all()
+
+
+@pytest.mark.parametrize("bits,group", [(8, 0), (4, 32), (4, 0), (4, 64)])
+def test_activations_on_the_int8_grid_give_the_fp16_activation_result_exactly(bits, group):
+    """If x is already scale * integer with |integer| <= 127 and the largest equal to 127, quantisation loses
+    nothing: the integer path must equal the plain linear layer's fp64 result exactly."""
+    N, K, M = 40, 256, 3
+    q, s = rand_layer(31, N, K, bits, group)
+    rng = np.random.default_rng(5)
+    ints = rng.integers(-127, 128, size=(M, K))
+    ints[:, 0] = 127
+    x = (ints * np.array([[2.0 ** -4], [2.0 ** -7], [2.0 ** 0]])).astype(np.float16)
+    y64, acc, xq, sx, _ = O.linear_int8_activations(x, q, s, group)
+    assert (xq == ints).all()
+    assert sx.tolist() == [2.0 ** -4, 2.0 ** -7, 1.0]
+    y_ref, _, _ = O.linear(x, q, s, group)
+    np.testing.assert_allclose(y64, y_ref, rtol=1e-13, atol=0)                      # same real number, fp64 summation order differs
+
+
+def test_integer_dot_products_are_exact_against_python_integers():
+    N, K, M, G = 5, 64, 2, 32
+    q, s = rand_layer(41, N, K, 4, G)
+    x = C.layer_activations(42, C.LayerSpec("t", N, K, 4, G, 0, 0), M)
+    y64, acc, xq, sx, _ = O.linear_int8_activations(x, q, s, G)
+    for m in range(M):
+        for n in range(N):
+            total = 0.0
+            for g in range(K // G):
+                a = sum(int(xq[m, k]) * int(q[n, k]) for k in range(g * G, (g + 1) * G))
+                assert a == int(acc[m, n, g])
+                total += float(s[n, g]) * a
+            assert abs(y64[m, n] - float(sx[m]) * total) <= 1e-12 * abs(y64[m, n]) + 1e-300
+
+
+def test_quantised_result_stays_close_to_the_unquantised_layer():
+    """A sign error, a dropped scale or a wrong group index would move the result by far more than int8 noise."""
+    N, K, M = 64, 2048, 4
+    q, s = rand_layer(51, N, K, 4, 32)
+    x = C.layer_activations(52, C.LayerSpec("t", N, K, 4, 32, 0, 0), M)
+    y64, _, _, _, _ = O.linear_int8_activations(x, q, s, 32)
+    y_ref, _, _ = O.linear(x, q, s, 32)
+    rel = np.linalg.norm(y64 - y_ref) / np.linalg.norm(y_ref)
+    assert 1e-4 < rel < 3e-2, rel
+
+
+# ----------------------------------------------------------------------------- KV cache as weights
+def test_example_H_kv_cache_orientation(golden):
+    e = golden["H_kv_cache"]
+    sc, _, _ = O.kv_scores(np.array(e["qry"], np.float16), np.array(e["k_q"], np.int8), np.array(e["k_s"], np.float16))
+    assert sc.tolist() == e["scores64"]
+    out, _, _ = O.kv_output(np.array(e["prob"], np.float16), np.array(e["v_q"], np.int8), np.array(e["v_s"], np.float16))
+    assert out.tolist() == e["out64"]
+
+
+def test_kv_products_against_plain_loops():
+    rng = np.random.default_rng(9)
+    T, d, R = 37, 16, 3
+    k_q = rng.integers(-128, 128, size=(T, d)).astype(np.int8)
+    k_s = rng.uniform(1e-3, 1e-2, size=T).astype(np.float16)
+    v_q = rng.integers(-128, 128, size=(d, T)).astype(np.int8)
+    v_s = rng.uniform(1e-3, 1e-2, size=d).astype(np.float16)
+    qry = rng.standard_normal((R, d)).astype(np.float16)
+    prob = rng.uniform(0, 1, size=(R, T)).astype(np.float16)
+    sc, _, _ = O.kv_scores(qry, k_q, k_s)
+    out, _, _ = O.kv_output(prob, v_q, v_s)
+    for r in range(R):
+        for t in range(T):                                   # one score per cached key: O = cache positions
+            want = sum(float(qry[r, j]) * float(k_s[t]) * int(k_q[t, j]) for j in range(d))
+            assert abs(sc[r, t] - want) <= 1e-12 * max(1.0, abs(want))
+        for j in range(d):                                   # one output per head dimension: O = d_h, I = cache positions
+            want = sum(float(prob[r, t]) * float(v_s[j]) * int(v_q[j, t]) for t in range(T))
+            assert abs(out[r, j] - want) <= 1e-12 * max(1.0, abs(want))

@@ -81,9 +81,19 @@ CONFIGS = (
 )
 CONFIG_5B = Workload("llama31_8b_lm_head", 5, (LLAMA31_8B_HEAD,), (1,), "decode")
 
+# The paper's two quantisation schemes on the same Llama3.1-8B shapes (Section 4.2: "q8" = int8 per channel
+# everywhere; "8/4/4" = int8 attention, int4 PER CHANNEL feed-forward), next to the benchmark's group-32 variant
+# (config 3).  Decode speed should follow the bytes: q8 streams 218.2 MB per pass, 8/4/4 per channel 130.1 MB.
+LLAMA31_8B_Q8 = tuple(_i8(l.name, l.N, l.K) for l in LLAMA31_8B)
+LLAMA31_8B_PC4 = tuple(l if l.bits == 8 else LayerSpec(l.name, l.N, l.K, 4, 0, -8, 7) for l in LLAMA31_8B)
+SCHEMES = (
+    Workload("llama31_8b_decode_q8", 6, LLAMA31_8B_Q8, (1,), "decode"),
+    Workload("llama31_8b_decode_pc4", 7, LLAMA31_8B_PC4, (1,), "decode"),
+)
+
 
 def by_name(name: str) -> Workload:
-    for w in CONFIGS + (CONFIG_5B,):
+    for w in CONFIGS + (CONFIG_5B,) + SCHEMES:
         if w.name == name:
             return w
     raise KeyError(name)
