@@ -584,12 +584,16 @@ def main():
 
     if rank == 0 and world == 1:
         if stage == "decode" and workload.name == "llama31_8b_decode":
+            # ---- every decode workload of the benchmark first, measured like the headline (the tensor-core legs
+            # that follow heat the part and would lower the clocks of whatever runs after them)
+            if not args.no_configs:
+                line["configs"] = decode_configs(torch, device, peaks, sidx, ls, line)
             # ---- second stage of the hot path on the SAME resident weights (copy 0), measured in the same run
             if not args.no_prefill:
                 line["prefill"] = prefill_sub(torch, device, peaks, args.prefill_steps, sidx, ls.blob0)
-            # ---- every workload of the benchmark, measured like the headline
             if not args.no_configs:
-                line["configs"] = all_configs(torch, device, peaks, sidx, ls, line)
+                line["configs"] += prefill_configs(torch, device, peaks, sidx, line)
+                line["fused_gating"] = gated_record(torch, device, peaks, sidx, ls)
         # ---- CPU oracle beside it (bounded sample)
         if not args.no_cpu_baseline:
             rows = calibrate_rows(workload, M, 8.0)
@@ -631,39 +635,81 @@ def prefill_sub(torch, device, peaks, steps, sidx, blobs):
     return out
 
 
-def all_configs(torch, device, peaks, sidx, ls_main, line):
-    """One entry per workload of the benchmark: the benchmark's five configs (config 3 at M = 1 and M = 4), the LM
-    head (5b), and the two schemes of the paper's Section 4.2 on the Llama shapes (q8; 8/4/4 per channel)."""
-    out = []
+def gated_record(torch, device, peaks, sidx, ls_main):
+    """The fused gating epilogue of the feed-forward block (paper Section 3.6) on the Llama gate / up layers,
+    next to the same two layers as one grouped call that writes both projections: decode at the headline's M,
+    prefill at M = 2048.  Same weights (the decode leg's resident copies), same x."""
+    import paper_2505_00232_b200 as P
+    w = ls_main.workload
+    ig = [i for i, l in enumerate(w.layers) if l.name == "gate"][0]
+    iu = [i for i, l in enumerate(w.layers) if l.name == "up"][0]
+    layer, act = w.layers[ig], "silu"
+    wbytes = layer.weight_bytes + w.layers[iu].weight_bytes
+    out = {"layers": f"gate, up {layer.N}x{layer.K} int{layer.bits} group {layer.group}", "act": act}
+    for stage, M in (("decode", ls_main.M), ("prefill", 2048)):
+        x = torch.from_numpy(C.layer_activations(w.seed, layer, M, ig)).to(device)
+        y = torch.empty((M, layer.N), dtype=torch.float16, device=device)
+        y2 = torch.empty((M, layer.N), dtype=torch.float16, device=device)
+        pairs = [(ls_main.lin[cp][ig], ls_main.lin[cp][iu]) for cp in range(ls_main.copies)]
+        fused = lambda cp: P.qlinear_forward_gated_raw(pairs[cp][0], pairs[cp][1], x.data_ptr(), y.data_ptr(), M, act)
+        plain = lambda cp: P.qlinear_forward_group_raw(list(pairs[cp]), x.data_ptr(), [y.data_ptr(), y2.data_ptr()], M)
+        rec = {"M": M}
+        for name, fn in (("gated", fused), ("grouped", plain)):
+            if stage == "decode":
+                graph = capture_graph(torch, lambda i: fn(i % ls_main.copies), ls_main.copies)
+                for _ in range(3):
+                    graph.replay()
+                ms, repeats, clocks = timed_region(torch, graph.replay, ls_main.copies, sidx, 0.25)
+            else:
+                def block():
+                    for cp in range(ls_main.copies):
+                        fn(cp)
+                block()
+                ms, repeats, clocks = timed_region(torch, block, ls_main.copies, sidx, 0.25)
+            rec[name + "_us"] = ms * 1e3 / (repeats * ls_main.copies)
+            rec[name + "_sm_mhz"] = clocks["sm_mhz"]
+        if stage == "decode":
+            rec["gated_gbs"] = wbytes / 1e3 / rec["gated_us"]
+            rec["gated_frac_of_measured_peak"] = rec["gated_gbs"] / peaks["hbm_gbs"]
+        else:
+            fl = layer.flops(M) + w.layers[iu].flops(M)
+            rec["gated_tflops"] = fl / 1e6 / rec["gated_us"]
+            rec["grouped_tflops"] = fl / 1e6 / rec["grouped_us"]
+            rec["y_bytes_written"] = {"gated": 2 * M * layer.N, "grouped": 4 * M * layer.N}
+        out[stage] = rec
+    return out
+
+
+def decode_configs(torch, device, peaks, sidx, ls_main, line):
+    """One entry per decode workload of the benchmark: the benchmark's configs 1-3 (config 3 at M = 1 and M = 4), the
+    LM head (5b), and the two schemes of the paper's Section 4.2 on the Llama shapes (q8; 8/4/4 per channel)."""
     main = {"workload": line["config"]["workload"], "M": line["config"]["M"], "metric": line["metric"], "value": line["value"],
             "unit": line["unit"], "us_per_step": line["ms_per_step"] * 1e3, "frac_of_measured_peak": line["frac_of_measured_peak"],
             "weight_bytes_per_step": ls_main.weight_bytes, "weight_copies": ls_main.copies, "launches_per_step": ls_main.launches_grouped,
             "steps": line["steps"], "repeats": line["repeats"], "timed_region_ms": line["timed_region_ms"], "clocks": line["clocks"],
             "gpu_launches": line["gpu_launches"], "note": "the headline of this line"}
-    # config 3 at M = 4 on the headline's four distinct weight copies
-    jobs = [("int8_gemv_2304", 1, {}), ("gemma2_2b_decode", 1, {})]
-    for name, M, kw in jobs:
-        out.append(config_entry(torch, device, peaks, sidx, name, M, **kw))
-    out.append(main)
-    out.append(config_entry(torch, device, peaks, sidx, "llama31_8b_decode", 4, copies=ls_main.copies, blobs=ls_main.blob0))
-    out.append(config_entry(torch, device, peaks, sidx, "gemma2_2b_prefill", 1024))
+    out = [config_entry(torch, device, peaks, sidx, "int8_gemv_2304", 1), config_entry(torch, device, peaks, sidx, "gemma2_2b_decode", 1), main,
+           config_entry(torch, device, peaks, sidx, "llama31_8b_decode", 4, copies=ls_main.copies, blobs=ls_main.blob0),
+           config_entry(torch, device, peaks, sidx, "llama31_8b_lm_head", 1)]
+    # the paper's schemes: bytes ratio and time ratio next to its "up to 1.9x" for decode (Section 4.2)
+    q8 = config_entry(torch, device, peaks, sidx, "llama31_8b_decode_q8", 1)
+    pc4 = config_entry(torch, device, peaks, sidx, "llama31_8b_decode_pc4", 1)
+    for e in (main, q8, pc4):
+        e["vs_q8"] = {"bytes_ratio": q8["weight_bytes_per_step"] / e["weight_bytes_per_step"],
+                      "time_ratio": q8["us_per_step"] / e["us_per_step"],
+                      "paper": "decode up to 1.9x faster with 8/4/4 than with q8 (Section 4.2; other hardware)"}
+    return out + [q8, pc4]
+
+
+def prefill_configs(torch, device, peaks, sidx, line):
+    """The prefill workloads: config 4 (Gemma2-2B FFN, M = 1024) and config 5 (the 'prefill' record of this line)."""
+    out = [config_entry(torch, device, peaks, sidx, "gemma2_2b_prefill", 1024)]
     if "prefill" in line and "value" in line["prefill"]:
         pf = line["prefill"]
         out.append({"workload": "llama31_8b_prefill", "M": pf["config"]["M"], "metric": pf["metric"], "value": pf["value"], "unit": pf["unit"],
                     "us_per_step": pf["ms_per_step"] * 1e3, "frac_of_measured_peak": pf["frac_of_measured_peak"],
                     "steps": pf["steps"], "repeats": pf["repeats"], "timed_region_ms": pf["timed_region_ms"], "clocks": pf["clocks"],
                     "gpu_launches": pf["gpu_launches"], "note": "same record as 'prefill'"})
-    out.append(config_entry(torch, device, peaks, sidx, "llama31_8b_lm_head", 1))
-    # the paper's schemes: bytes ratio and time ratio next to its "up to 1.9x" for decode (Section 4.2)
-    q8 = config_entry(torch, device, peaks, sidx, "llama31_8b_decode_q8", 1)
-    pc4 = config_entry(torch, device, peaks, sidx, "llama31_8b_decode_pc4", 1)
-    for e in (q8, pc4):
-        e["vs_q8"] = {"bytes_ratio": q8["weight_bytes_per_step"] / e["weight_bytes_per_step"],
-                      "time_ratio": q8["us_per_step"] / e["us_per_step"],
-                      "paper": "decode up to 1.9x faster with 8/4/4 than with q8 (Section 4.2; other hardware)"}
-    main["vs_q8"] = {"bytes_ratio": q8["weight_bytes_per_step"] / main["weight_bytes_per_step"],
-                     "time_ratio": q8["us_per_step"] / main["us_per_step"]}
-    out += [q8, pc4]
     return out
 
 

@@ -132,6 +132,28 @@ ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
 
+/* Activation of the gate branch in qlinear_forward_gated. */
+typedef enum { QL_ACT_IDENTITY = 0, QL_ACT_SILU = 1, QL_ACT_GELU_TANH = 2 } ql_act;
+
+/* Fused gating of the feed-forward block (Section 3.6, "Operator Fusion": element-wise operators of two
+ * branches fused with a fully connected operator):
+ *     y[m,n] = fp16( act(gate[m,n]) * up[m,n] ),   gate = x . W_gate^T,  up = x . W_up^T   (both in fp32)
+ * with act = identity, SiLU g / (1 + exp(-g)) (the Llama family) or the tanh form of GELU (the Gemma family);
+ * the paper names no activation.  Neither projection is written to memory: for M <= 8 one decode launch
+ * holds both branches of every output channel in the same CTA; for M > 128 (and layers of a multiple of 256
+ * channels after padding to 128) the CTA-pair prefill kernel keeps the two projections of a tile in its two
+ * tensor-memory accumulators and the epilogue writes only their product, which halves the write-back.
+ * Shapes outside those two cases (9 <= M <= 128, other channel counts, K not a multiple of the decode chunk)
+ * run the two projections into the device's shared scratch and a small element-wise kernel after them: same
+ * result, no saving; such calls must be ordered against K-split prefill calls like those among themselves.
+ *   h_gate, h_up  two layers on one device with the same N, K, bits and group
+ *   x_dev, y_dev  as in qlinear_forward; y_dev is fp16 [M, N]
+ * Asynchronous, allocates nothing.  Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for layers that do
+ * not agree or an unknown activation; QL_ERR_UNSUPPORTED if the unfused case needs more scratch than the
+ * device's shared buffer holds (2 * M * N fp16 beyond about 19 MB). */
+ql_status qlinear_forward_gated(qlinear_t h_gate, qlinear_t h_up, const void* x_dev, void* y_dev, int32_t M,
+                                int32_t act, void* cuda_stream);
+
 /* Embedding lookup from a quantised table (Section 4.2: the mixed 8/4/4 scheme keeps the embedding table
  * in int4 like the feed-forward weights).  The handle's layer is read as a table of N rows of K values:
  *   y_dev[t, k] = fp16( s[ids[t], k / group] * q[ids[t], k] )      for t in [0, n), k in [0, K)

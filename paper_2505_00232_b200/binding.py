@@ -18,9 +18,11 @@ LIB_PATH = os.path.join(_HERE, "libqlinear.so")
 QL_OK = 0
 QL_ERR_INVALID_ARG, QL_ERR_UNSUPPORTED, QL_ERR_ALLOC, QL_ERR_CUDA, QL_ERR_DEVICE_TIMEOUT, QL_ERR_ARCH = 1, 2, 3, 4, 5, 6
 QL_PATH_GEMV, QL_PATH_GEMM = 1, 2
+QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
+ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_embed",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_embed",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -60,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_debug_unpack_device.restype = ctypes.c_int
     lib.qlinear_forward_group.argtypes = [ctypes.POINTER(vp), ctypes.c_int32, vp, ctypes.POINTER(vp), ctypes.c_int32, vp]
     lib.qlinear_forward_group.restype = ctypes.c_int
+    lib.qlinear_forward_gated.argtypes = [vp, vp, vp, vp, i32, i32, vp]
+    lib.qlinear_forward_gated.restype = ctypes.c_int
     lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
     lib.qlinear_embed.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
@@ -189,6 +193,28 @@ def qlinear_forward_group(lins, x, outs=None, stream=None):
             raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_group (bad out tensor)")
     qlinear_forward_group_raw(lins, x.data_ptr(), [o.data_ptr() for o in outs], M, stream)
     return outs
+
+
+def qlinear_forward_gated_raw(gate, up, x_ptr: int, y_ptr: int, M: int, act: str, stream=None) -> None:
+    _check(lib.qlinear_forward_gated(gate._h, up._h, ctypes.c_void_p(x_ptr), ctypes.c_void_p(y_ptr), M, ACTIVATIONS[act],
+                                     _stream_ptr(stream)), "qlinear_forward_gated")
+
+
+def qlinear_forward_gated(gate, up, x, act: str = "silu", out=None, stream=None):
+    """y = act(x . W_gate^T) * (x . W_up^T) as fp16 [M, N], from one fused launch where the shape allows."""
+    import torch
+    K, N = gate.desc.K, gate.desc.N
+    if x.dim() != 2 or x.shape[1] != K or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_gated (x must be contiguous fp16 CUDA [M, K])")
+    if act not in ACTIVATIONS:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_gated (unknown activation)")
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float16, device=x.device)
+    elif out.shape != (M, N) or out.dtype != torch.float16 or not out.is_contiguous():
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_gated (bad out tensor)")
+    qlinear_forward_gated_raw(gate, up, x.data_ptr(), out.data_ptr(), M, act, stream)
+    return out
 
 
 class QLinear:

@@ -9,7 +9,35 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "../../include/qlinear.h"
+
 namespace ql {
+
+// Activation of the gate branch in the fused gating epilogue (paper Section 3.6), fp32, with the hardware
+// exponential and reciprocal (a few ulp, far inside the tolerance of the product).
+// tanh(t) = 1 - 2 / (exp(2t) + 1), so 0.5 * g * (1 + tanh(t)) = g * (1 - 1 / (exp(2t) + 1)) = g / (1 + exp(-2t)).
+__device__ __forceinline__ float gate_activation(float g, int act)
+{
+    if (act == QL_ACT_IDENTITY) return g;
+    const float t = act == QL_ACT_SILU ? g : 1.5957691216057308f * (g + 0.044715f * g * g * g);
+    return __fdividef(g, 1.f + __expf(-t));
+}
+
+// mma.m16n8k16 (fp16 in, fp32 accumulate), not `volatile`: the compiler may interleave independent MMA chains.
+__device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+// D = A.B with a zero accumulator input (no register has to be cleared first).
+__device__ __forceinline__ void mma_16816_zero(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
+{
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
 
 __device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t mask, uint32_t orv)
 {

@@ -60,6 +60,7 @@ struct GemmParams {
     int32_t lN[4];
     int32_t rsb_end[4];
     int32_t n_layers;
+    int32_t act;                             // pair kernel, gated form: activation of the gate branch (QL_ACT_*)
 };
 constexpr int kGemmMaxGroup = 4;
 

@@ -72,10 +72,17 @@ __device__ __forceinline__ int pair_layer(const GemmParams& p, int& rsb)
     return ly;
 }
 
-template <int BITS, bool GROUPED, int TB>
+// GATED (TB == 1 only): the launch serves two layers of equal shape, gate (0) and up (1).  A cluster runs the gate
+// tile and the up tile of the same (row super-block pair, token block) back to back into its two accumulators.
+// While the up tile's main loop runs, the epilogue warps turn the finished gate accumulator into act(gate) in
+// place (tensor memory load, activation, tensor memory store); when the up tile is complete they write
+// fp16(act(gate) * up), the only tensor that ever goes to memory (paper Section 3.6), and free both accumulators.
+// Work unit t then counts (row super-block pair, token block) positions of ONE layer; every unit is two tiles.
+template <int BITS, bool GROUPED, int TB, bool GATED = false>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
+    static_assert(!GATED || TB == 1, "the gated form uses both accumulators for one output tile");
     using S = GemmPairSmem<BITS, TB>;
     constexpr int NS = S::kStages;
     constexpr int NA = S::kASlots;
@@ -105,6 +112,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     // weight blocks and read different x tiles, which spreads the L2 traffic over more lines.
     const int n_mblk = (p.M + TILE_N - 1) / TILE_N;
     const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
+    // The j-th tile this cluster runs: work unit t and, in the gated form, which of the two layers.
+    auto tile_of = [&](int j, int& t, int& gl) {
+        t = first_tile + (GATED ? j >> 1 : j) * tile_stride;
+        gl = GATED ? (j & 1) : 0;
+        return t < p.n_tiles;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < NS; ++s) {
@@ -139,11 +152,12 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             int s = 0, issued = 0;
             uint32_t par = 1;
             bool waited_dep = false, ok = true;
-            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+            int t, gl;
+            for (int j = 0; tile_of(j, t, gl) && ok; ++j) {
                 const PairUnit u = pair_unit(t, p);
                 const int tile = u.tile, step0 = u.step0, n_steps = u.nsteps;
                 int rsb = 2 * (tile / n_mblk) + (int)rank;
-                const int ly = pair_layer(p, rsb);
+                const int ly = GATED ? gl : pair_layer(p, rsb);
                 const int m0 = (tile % n_mblk) * TILE_N + 128 * (int)rank;   // this CTA's 128 tokens of each token block
                 const uint8_t* wsrc = p.lbody[ly] + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
@@ -179,8 +193,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             int s = 0, a = 0;
             uint32_t apar = 0;
             bool ok = true;
-            int j = 0;
-            for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+            int t, gl;
+            for (int j = 0; tile_of(j, t, gl) && ok; ++j) {
                 // TB = 1: two accumulators alternate; TB = 2: both are used by every tile
                 const int buf = TB == 1 ? (j & 1) : 0;
                 const uint32_t use = TB == 1 ? (uint32_t)(j >> 1) : (uint32_t)j;
@@ -222,7 +236,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             if (rank != 0 && lane == 0 && a < NA) {
                 uint32_t apar = 0;
                 int total_steps = 0;
-                for (int t = first_tile; t < p.n_tiles; t += tile_stride) total_steps += pair_unit(t, p).nsteps;
+                int t, gl;
+                for (int j = 0; tile_of(j, t, gl); ++j) total_steps += pair_unit(t, p).nsteps;
                 for (int g = a; g < total_steps; g += NA) {
                     if (!mbar_wait(afull_bar(a), apar, abort_flag, 0xA00 + a)) break;
                     mbar_arrive_remote(afull_bar(a), 0);
@@ -239,7 +254,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         uint32_t par_old = 0;
         bool ok = true;
         int gstep = 0;
-        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride) {
+        int t, gl;
+        for (int j = 0; tile_of(j, t, gl) && ok; ++j) {
             const int n_steps = pair_unit(t, p).nsteps;
             for (int it = 0; it < n_steps; ++it, ++gstep) {
                 if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
@@ -260,18 +276,56 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ------------------------------------------------------------------ epilogue (each CTA stores its 128 channels)
         const int quarter = warp & 3;
         bool ok = true;
-        int j = 0;
-        for (int t = first_tile; t < p.n_tiles && ok; t += tile_stride, ++j) {
+        int t, gl;
+        for (int j = 0; tile_of(j, t, gl) && ok; ++j) {
             const int buf = TB == 1 ? (j & 1) : 0;
             const uint32_t use = TB == 1 ? (uint32_t)(j >> 1) : (uint32_t)j;
             const PairUnit u = pair_unit(t, p);
             const int tile = u.tile, part = u.part;
             int rsb = 2 * (tile / n_mblk) + (int)rank;
-            const int ly = pair_layer(p, rsb);
+            const int ly = GATED ? 0 : pair_layer(p, rsb);
             const int m0 = (tile % n_mblk) * TILE_N, N = p.lN[ly];
             if (!mbar_wait<true>(tfull_bar(buf), use & 1, abort_flag, 0x500 + buf)) { ok = false; break; }
             tc_fence_after();
             const int n = rsb * kRsbRows + quarter * 32 + lane;
+            if (GATED) {
+                // accumulator 0 holds the gate projection of this tile, accumulator 1 the up projection
+                float sg = 1.f, su = 1.f;
+                if (!GROUPED && n < N) { sg = __half2float(p.lscales[0][n]); su = __half2float(p.lscales[1][n]); }
+                const uint32_t tg = tmem_base + ((uint32_t)(quarter * 32) << 16);
+                const int m_left = min(TILE_N, p.M - m0);
+                if (gl == 0) {
+                    // The gate accumulator is complete while the up tile's main loop runs: apply scale and activation
+                    // in place now, so that only a product is left to do once the up tile is complete.
+#pragma unroll 1
+                    for (int cc = 0; cc < m_left; cc += 16) {
+                        uint32_t rg[16];
+                        tmem_ld16(tg + (uint32_t)cc, rg);
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) rg[q] = __float_as_uint(gate_activation(__uint_as_float(rg[q]) * sg, p.act));
+                        tmem_st16(tg + (uint32_t)cc, rg);
+                    }
+                    tc_fence_before();
+                    continue;
+                }
+                __half* yrow = p.ly[0] + (int64_t)m0 * N + n;
+#pragma unroll 1
+                for (int cc = 0; cc < m_left; cc += 16) {
+                    uint32_t rg[16], ru[16];
+                    tmem_ld16(tg + (uint32_t)cc, rg);
+                    tmem_ld16(tg + (uint32_t)(BN + cc), ru);
+                    if (n < N) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            if (cc + q < m_left)
+                                yrow[(int64_t)(cc + q) * N] = __float2half_rn(__uint_as_float(rg[q]) * (__uint_as_float(ru[q]) * su));
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive_remote(tempty_bar(0), 0); mbar_arrive_remote(tempty_bar(1), 0); }
+                continue;
+            }
             float scale = 1.f;
             if (!GROUPED && n < N) scale = __half2float(p.lscales[ly][n]);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
@@ -387,15 +441,16 @@ struct GemmPairLayers {
     int n_rsb() const { int t = 0; for (int i = 0; i < n; ++i) t += L[i]->n_rsb; return t; }
 };
 
-template <int BITS, bool GROUPED, int TB>
+// act < 0: the plain form.  act >= 0 (TB == 1): the gated form, set = {gate, up} of equal shape, y[0] the output.
+template <int BITS, bool GROUPED, int TB, bool GATED = false>
 ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device,
-                           bool pdl, int num_sms, float* scratch, unsigned int* counters)
+                           bool pdl, int num_sms, float* scratch, unsigned int* counters, int act = -1)
 {
     using S = GemmPairSmem<BITS, TB>;
     const Layout& L = *set.L[0];
     CUtensorMap map;
     if (!x_tensor_map(x, L.K, M, 128, &map)) return QL_ERR_CUDA;
-    auto kern = gemm_pair_kernel<BITS, GROUPED, TB>;
+    auto kern = gemm_pair_kernel<BITS, GROUPED, TB, GATED>;
     static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
@@ -416,6 +471,8 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
         prm.rsb_end[i] = n_rsb;
     }
     prm.n_layers = set.n;
+    prm.act = act;
+    if (GATED) n_rsb = L.n_rsb;                                          // work units count positions of one layer
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
@@ -426,7 +483,7 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
     // (splitting the tail of a multi-round schedule was measured and does not pay: the exposed scratch
     // reduction costs what the shorter last round saves; only single-round layers are split)
     const int tail = tiles < clusters ? tiles : 0;
-    prm.split = TB == 1 ? gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr) : 1;
+    prm.split = (TB == 1 && !GATED) ? gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr) : 1;
     prm.n_whole = prm.split > 1 ? tiles - tail : tiles;
     prm.scratch = scratch;
     prm.counters = counters;
@@ -482,6 +539,16 @@ inline ql_status gemm_pair_forward(const GemmPairLayers& set, const void* x, int
     if (L.bits == 8) return gemm_pair_launch<8, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
     if (L.grouped) return gemm_pair_launch<4, true, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
     return gemm_pair_launch<4, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+}
+
+// Gated form: set = {gate, up}, both pair-applicable and of equal shape; y[0] receives act(gate) * up.
+inline ql_status gemm_pair_forward_gated(const GemmPairLayers& set, const void* x, int M, int act, cudaStream_t st,
+                                         int device, bool pdl, int num_sms)
+{
+    const Layout& L = *set.L[0];
+    if (L.bits == 8) return gemm_pair_launch<8, false, 1, true>(set, x, M, st, device, pdl, num_sms, nullptr, nullptr, act);
+    if (L.grouped) return gemm_pair_launch<4, true, 1, true>(set, x, M, st, device, pdl, num_sms, nullptr, nullptr, act);
+    return gemm_pair_launch<4, false, 1, true>(set, x, M, st, device, pdl, num_sms, nullptr, nullptr, act);
 }
 
 }  // namespace ql

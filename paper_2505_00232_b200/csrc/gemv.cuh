@@ -50,25 +50,14 @@ struct GemvParams {
     int32_t cps;                         // chunks per slice
     int32_t x_stride;                    // halves between tokens in the shared x slab
     int32_t x_bytes;                     // bytes of the x slab (the warp rings follow it)
+    int32_t act;                         // gated form only: activation of the gate branch (QL_ACT_*)
 };
 
-// mma.m16n8k16 (fp16 in, fp32 accumulate), not `volatile`: the compiler may interleave independent MMA chains.
-__device__ __forceinline__ void mma_16816_pure(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
-{
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-
-// D = A.B with a zero accumulator input (no register has to be cleared first).
-__device__ __forceinline__ void mma_16816_zero(float d[4], const uint32_t a[4], uint32_t b0, uint32_t b1)
-{
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
-}
-
-template <int BITS, bool GROUPED, bool XDIRECT>
+// GATED: the launch serves exactly two layers of equal shape, gate (0) and up (1), whose row-blocks are dealt out
+// alternately, so that a CTA (which then holds an even number of row-blocks, no cluster) has both branches of
+// every output channel it owns; the epilogue writes y[0] = act(gate) * up (paper Section 3.6: element-wise
+// operators of two branches fused with a fully connected operator).
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false>
 __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -91,10 +80,13 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     const int rb_all = rb_group * rb_per_cta + (warp >> p.ks_cta_log2);  // numbered through all layers of the launch
     const bool rb_live = rb_all < p.n_rb;
     int layer = 0;
+    if (GATED) layer = rb_all & 1;
+    else {
 #pragma unroll
-    for (int i = 1; i < kGemvMaxGroup; ++i)
-        if (i < p.n_layers && rb_all >= p.rb_end[i - 1]) layer = i;
-    const int rb = rb_all - (layer ? p.rb_end[layer - 1] : 0);           // row-block inside its layer
+        for (int i = 1; i < kGemvMaxGroup; ++i)
+            if (i < p.n_layers && rb_all >= p.rb_end[i - 1]) layer = i;
+    }
+    const int rb = GATED ? rb_all >> 1 : rb_all - (layer ? p.rb_end[layer - 1] : 0);   // row-block inside its layer
     const int ks = crank * p.ks_cta + ks_local;
     const int kc0 = min(ks * p.cps, p.n_kc);
     const int kc1 = rb_live ? min(kc0 + p.cps, p.n_kc) : kc0;
@@ -298,6 +290,19 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             store_out(0, t, v);
         }
         cluster.sync();                                                  // peers keep `part` alive until read
+    } else if (GATED) {
+        for (int idx = t; idx < (rb_per_cta >> 1) * 128; idx += kGemvThreads) {
+            const int pr = idx >> 7, e = idx & 127;                      // pair of row-blocks (gate, up), element
+            float gv = 0.f, uv = 0.f;
+            for (int s = 0; s < p.ks_cta; ++s) { gv += red[(2 * pr) * p.ks_cta + s][e]; uv += red[(2 * pr + 1) * p.ks_cta + s][e]; }
+            const int out_rb = ((rb_group * rb_per_cta) >> 1) + pr;
+            const int el = e >> 2, i = e & 3;
+            const int row = out_rb * kRbRows + (el >> 2) + 8 * (i >> 1), tok = 2 * (el & 3) + (i & 1);
+            if (row < p.N[0] && tok < p.M) {
+                if (!GROUPED) { gv *= __half2float(p.chan_scales[0][row]); uv *= __half2float(p.chan_scales[1][row]); }
+                p.y[0][(int64_t)tok * p.N[0] + row] = __float2half_rn(gate_activation(gv, p.act) * uv);
+            }
+        }
     } else {
         for (int idx = t; idx < rb_per_cta * 128; idx += kGemvThreads) {
             const int rbl = idx >> 7, e = idx & 127;

@@ -133,7 +133,8 @@ namespace {
 constexpr int kGemvMaxSmem = 96 * 1024;
 
 // n_rb: row-blocks of the launch (one layer, or all layers of a group that shares x).
-GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
+// gated: the launch needs both branches of a channel in one CTA: an even number of row-blocks per CTA, no cluster.
+GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = false)
 {
     const Config& cfg = config();
     const double target = (double)num_sms * cfg.warps_per_sm;
@@ -141,6 +142,7 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
     double best_score = -1e30;
     for (int ks_cta = 1; ks_cta <= 8; ks_cta *= 2)
         for (int cl = 1; cl <= (ks_cta == 8 ? 8 : 1); ++cl) {
+            if (gated && (ks_cta > 4 || cl > 1)) continue;
             const int ks = ks_cta * cl;
             const int cps = (L.n_kc + ks - 1) / ks;
             if ((ks - 1) * cps >= L.n_kc && ks > 1) continue;               // would leave a slice empty
@@ -158,7 +160,7 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms)
             // slices on half as many warps)
             double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 4 ? 1.25 : 0.0) - (cps < 2 ? 1.0 : 0.0);
             if (warps > target) score -= 2.0;                               // more CTAs than fit at once: a second wave
-            if (cfg.force_ks) score = (ks == cfg.force_ks) ? 0.0 : -1e29;
+            if (cfg.force_ks && !gated) score = (ks == cfg.force_ks) ? 0.0 : -1e29;
             if (score > best_score) {
                 best_score = score;
                 const int rb_per_cta = kGemvWarps / ks_cta;
@@ -210,32 +212,37 @@ cudaError_t ensure_smem_attr(Kern kern, std::atomic<bool>* flags, int device, in
     return e;
 }
 
-template <int BITS, bool GROUPED, bool XDIRECT>
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false>
 cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
 {
     static std::atomic<bool> attr_set[kMaxDevices];
-    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT>;
+    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT, GATED>;
     cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, kGemvMaxSmem);
     if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
 }
 
 template <int BITS, bool GROUPED>
-cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
+cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st, bool gated = false)
 {
+    if (gated) return launch_gemv_x<BITS, GROUPED, true, true>(h, prm, pl, st);     // (planned only with direct x)
     return prm.x_bytes == 0 ? launch_gemv_x<BITS, GROUPED, true>(h, prm, pl, st)
                             : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
 }
 
 // One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
 // call (integer arithmetic only); nothing is written to a handle.
-ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st)
+// act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
+ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1)
 {
     const qlinear_s* h = hs[0];
     const Layout& L = h->L;
     int n_rb = 0;
     for (int i = 0; i < n; ++i) n_rb += hs[i]->n_rb;
-    const GemvPlan pl = n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
+    const bool gated = act >= 0;
+    if (gated) n_rb = 2 * hs[0]->n_rb;
+    const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
+    if (gated && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
     cudaError_t e;
     if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
     GemvParams prm{};
@@ -244,22 +251,31 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
         const Layout& Li = hs[i]->L;
         prm.body[i] = hs[i]->blob + Li.body_offset;
         prm.chan_scales[i] = Li.grouped ? nullptr : reinterpret_cast<const __half*>(hs[i]->blob + Li.chan_scale_offset);
-        prm.y[i] = static_cast<__half*>(ys[i]);
+        prm.y[i] = static_cast<__half*>(ys[gated ? 0 : i]);
         prm.N[i] = Li.N;
         acc += hs[i]->n_rb;
         prm.rb_end[i] = acc;
     }
     prm.n_layers = n;
+    prm.act = gated ? act : 0;
     prm.x = static_cast<const __half*>(x);
     prm.M = M; prm.K = L.K;
     prm.n_rb = n_rb;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
-    if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st);
-    else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st);
-    else e = launch_gemv<4, false>(h, prm, pl, st);
+    if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st, gated);
+    else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st, gated);
+    else e = launch_gemv<4, false>(h, prm, pl, st, gated);
     return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+// y = act(g) * u, element-wise (the unfused form of the gating, for shapes the fused kernels do not take).
+__global__ void __launch_bounds__(256) gate_mul_kernel(const __half* g, const __half* u, __half* y, int64_t n, int act)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256)
+        y[i] = __float2half_rn(gate_activation(__half2float(g[i]), act) * __half2float(u[i]));
 }
 
 template <int BITS, bool GROUPED, int NS>
@@ -522,6 +538,43 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         if (s != QL_OK) return s;
     }
     return QL_OK;
+}
+
+extern "C" ql_status qlinear_forward_gated(qlinear_t hg, qlinear_t hu, const void* x, void* y, int32_t M, int32_t act, void* stream)
+{
+    if (!hg || !hu || !x || !y || M < 1) return QL_ERR_INVALID_ARG;
+    if (act != QL_ACT_IDENTITY && act != QL_ACT_SILU && act != QL_ACT_GELU_TANH) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
+    const Layout &a = hg->L, &b = hu->L;
+    if (hg->device != hu->device || a.N != b.N || a.K != b.K || a.bits != b.bits || a.group != b.group) return QL_ERR_INVALID_ARG;
+    if ((int64_t)M * a.K > INT32_MAX || (int64_t)M * a.N > INT32_MAX) return QL_ERR_INVALID_ARG;
+    if (device_timed_out(hg)) return QL_ERR_DEVICE_TIMEOUT;
+    DeviceGuard guard(hg->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    qlinear_s* hs[2] = {hg, hu};
+    if (M <= hg->gemv_max_m && !hg->use_stream) {                        // decode: both branches in one launch
+        void* ys[2] = {y, y};
+        const ql_status s = forward_gemv(hs, 2, x, ys, M, st, act);
+        if (s != QL_ERR_UNSUPPORTED) return s;
+    } else if (M > hg->gemv_max_m && gemm_pair_applicable(a, M)) {       // prefill: both accumulators of the CTA-pair kernel
+        GemmPairLayers set{};
+        set.n = 2;
+        set.L[0] = &hg->L; set.blob[0] = hg->blob; set.y[0] = y;
+        set.L[1] = &hu->L; set.blob[1] = hu->blob; set.y[1] = y;
+        return gemm_pair_forward_gated(set, x, M, act, st, hg->device, hg->pdl, hg->num_sms);
+    }
+    // Unfused: the two projections into the device's shared scratch, then the element-wise product.
+    const int64_t n = (int64_t)M * a.N;
+    if ((size_t)n * 2 * sizeof(__half) > gemm_pair_scratch_bytes(hg->num_sms)) return QL_ERR_UNSUPPORTED;
+    __half* g = reinterpret_cast<__half*>(hg->dev->gemm_scratch);
+    __half* u = g + ((n + 7) & ~(int64_t)7);
+    void* ys[2] = {g, u};
+    ql_status s = qlinear_forward_group(hs, 2, x, ys, M, stream);
+    if (s != QL_OK) return s;
+    const int blocks = (int)std::min<int64_t>((n + 255) / 256, (int64_t)hg->num_sms * 8);
+    gate_mul_kernel<<<blocks, 256, 0, st>>>(g, u, static_cast<__half*>(y), n, act);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
 extern "C" ql_status qlinear_embed(qlinear_t h, const int32_t* ids, int32_t n, void* y, void* stream)
