@@ -161,7 +161,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 const int m0 = (tile % n_mblk) * TILE_N + 128 * (int)rank;   // this CTA's 128 tokens of each token block
                 const uint8_t* wsrc = p.lbody[ly] + (int64_t)rsb * p.n_kc * p.block_bytes;
                 for (int it = 0; it < n_steps; ++it) {
-                    if (!mbar_wait<true>(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
+                    if (!mbar_wait_hot(empty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
                     const int kc = (step0 + it) * CHUNKS;
                     const int nblk = min(CHUNKS, p.n_kc - kc);
                     const uint32_t wbytes = (uint32_t)nblk * p.block_bytes;
@@ -205,7 +205,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 for (int it = 0; it < n_steps; ++it) {
                     // own A tile written (implies own x half landed) and the peer's likewise
                     // 16 local dequantise warps + the peer's relay lane: both A tiles written, both x halves landed
-                    if (!mbar_wait(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
+                    if (!mbar_wait_hot(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);

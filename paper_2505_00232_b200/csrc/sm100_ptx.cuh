@@ -55,6 +55,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// Bounded hot wait: polls without a suspend hint or back-off, for the single threads on the critical path of a
+// pipeline (the MMA issuer, the TMA producer), whose wake-up latency is paid on every step.
+__device__ __forceinline__ bool mbar_wait_hot(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t code)
+{
+    auto test = [&]() {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        return ok != 0;
+    };
+    if (test()) return true;
+    long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 128; ++i)
+            if (test()) return true;
+        if (*abort_flag) return false;
+        if (wait_expired(t0, abort_flag)) {
+            report_timeout(abort_flag, code);
+            return false;
+        }
+    }
+}
+
 // Bounded wait.  Returns false if the wait expired or another thread of the CTA already gave up.
 // SLEEP: back off between polls (for waits that are long and off the critical path, so that the issue
 // slots go to warps that have work); without it the wait wakes up as soon as the phase completes.
