@@ -154,6 +154,27 @@ typedef enum { QL_ACT_IDENTITY = 0, QL_ACT_SILU = 1, QL_ACT_GELU_TANH = 2 } ql_a
 ql_status qlinear_forward_gated(qlinear_t h_gate, qlinear_t h_up, const void* x_dev, void* y_dev, int32_t M,
                                 int32_t act, void* cuda_stream);
 
+/* The linear layer with int8 ACTIVATIONS, decode stage (Section 3.7, "Stage-Aware Optimizations": in the
+ * memory-bound decode stage the quantisation of the input activations is integrated into the fully-connected
+ * kernel, the products with the pre-quantised weights use integer instructions, and the dequantisation is
+ * applied to the output).  Per token m:  amax = max_k |x[m,k]|,  xq = round-half-to-even(x * (127 / amax))
+ * clamped to [-127, 127] (IEEE fp32, one rounding per operation; a row of zeros quantises to zeros with scale 1),
+ *     y[m,n] = fp16( (amax / 127) * sum_g s[n,g] * sum_{k in g} xq[m,k] * q[n,k] )
+ * with the inner sums exact (integer tensor-core instructions).  The paper gives neither the granularity of the
+ * activation scale nor the rounding; one scale per token, symmetric, is the reading taken here.
+ *   h, x_dev, y_dev, cuda_stream as in qlinear_forward;  1 <= M <= 8 (QL_ERR_UNSUPPORTED beyond: the prefill
+ *   form -- qlinear_quantize_activations followed by an integer matmul -- has only its first kernel so far).
+ * Asynchronous, allocates nothing.  The result differs from qlinear_forward's by the quantisation noise of x
+ * (about 1 % relative for Gaussian x); it equals it to fp32 round-off when x already lies on the int8 grid. */
+ql_status qlinear_forward_a8(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
+
+/* The activation-quantisation kernel of the prefill stage (Section 3.7): x_dev fp16 [M, K] -> xq_dev int8 [M, K]
+ * and scale_dev fp32 [M], by the per-token steps stated at qlinear_forward_a8.  K a multiple of 32; x_dev and
+ * xq_dev 16-byte aligned; all three buffers on `device`, caller-owned.  Asynchronous on `cuda_stream`.
+ * Errors: QL_ERR_INVALID_ARG, QL_ERR_CUDA. */
+ql_status qlinear_quantize_activations(const void* x_dev, int8_t* xq_dev, float* scale_dev, int32_t M, int32_t K,
+                                       int device, void* cuda_stream);
+
 /* Embedding lookup from a quantised table (Section 4.2: the mixed 8/4/4 scheme keeps the embedding table
  * in int4 like the feed-forward weights).  The handle's layer is read as a table of N rows of K values:
  *   y_dev[t, k] = fp16( s[ids[t], k / group] * q[ids[t], k] )      for t in [0, n), k in [0, K)

@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_embed",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_embed",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -64,6 +64,10 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_forward_group.restype = ctypes.c_int
     lib.qlinear_forward_gated.argtypes = [vp, vp, vp, vp, i32, i32, vp]
     lib.qlinear_forward_gated.restype = ctypes.c_int
+    lib.qlinear_forward_a8.argtypes = [vp, vp, vp, i32, vp]
+    lib.qlinear_forward_a8.restype = ctypes.c_int
+    lib.qlinear_quantize_activations.argtypes = [vp, vp, vp, i32, i32, ctypes.c_int, vp]
+    lib.qlinear_quantize_activations.restype = ctypes.c_int
     lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
     lib.qlinear_embed.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
@@ -217,6 +221,19 @@ def qlinear_forward_gated(gate, up, x, act: str = "silu", out=None, stream=None)
     return out
 
 
+def qlinear_quantize_activations(x, stream=None):
+    """x fp16 CUDA [M, K] -> (xq int8 [M, K], scale fp32 [M]): the prefill stage's quantisation kernel."""
+    import torch
+    if x.dim() != 2 or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous() or x.shape[1] % 32:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_quantize_activations (x must be contiguous fp16 CUDA [M, K], K % 32 == 0)")
+    M, K = x.shape
+    xq = torch.empty((M, K), dtype=torch.int8, device=x.device)
+    scale = torch.empty((M,), dtype=torch.float32, device=x.device)
+    _check(lib.qlinear_quantize_activations(ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(xq.data_ptr()), ctypes.c_void_p(scale.data_ptr()),
+                                            M, K, x.device.index or 0, _stream_ptr(stream)), "qlinear_quantize_activations")
+    return xq, scale
+
+
 class QLinear:
     """One quantised linear layer resident on a GPU: owns the packed device tensor and the handle."""
 
@@ -253,6 +270,20 @@ class QLinear:
         elif out.shape != (M, self.desc.N) or out.dtype != torch.float16 or not out.is_contiguous():
             raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward (bad out tensor)")
         self.forward_raw(x.data_ptr(), out.data_ptr(), M, stream)
+        return out
+
+    def forward_a8(self, x, out=None, stream=None):
+        """The decode call with int8 activations quantised inside the kernel (qlinear_forward_a8), M <= 8."""
+        import torch
+        if x.dim() != 2 or x.shape[1] != self.desc.K or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_a8 (x must be contiguous fp16 CUDA [M, K])")
+        M = x.shape[0]
+        if out is None:
+            out = torch.empty((M, self.desc.N), dtype=torch.float16, device=x.device)
+        elif out.shape != (M, self.desc.N) or out.dtype != torch.float16 or not out.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_a8 (bad out tensor)")
+        _check(lib.qlinear_forward_a8(self._h, ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(out.data_ptr()), M, _stream_ptr(stream)),
+               "qlinear_forward_a8")
         return out
 
     def forward_raw(self, x_ptr: int, y_ptr: int, M: int, stream=None) -> None:

@@ -26,6 +26,7 @@ __device__ unsigned int* g_status_host;
 #include "embed.cuh"
 #include "gemv.cuh"
 #include "gemv_stream.cuh"
+#include "gemv_a8.cuh"
 #include "gemm.cuh"
 #include "gemm_pair.cuh"
 
@@ -134,7 +135,8 @@ constexpr int kGemvMaxSmem = 96 * 1024;
 
 // n_rb: row-blocks of the launch (one layer, or all layers of a group that shares x).
 // gated: the launch needs both branches of a channel in one CTA: an even number of row-blocks per CTA, no cluster.
-GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = false)
+// a8: the int8-activation kernel keeps the quantised x of the CTA's K range, and its per-group sums, in shared memory.
+GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = false, bool a8 = false)
 {
     const Config& cfg = config();
     const double target = (double)num_sms * cfg.warps_per_sm;
@@ -151,7 +153,9 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = f
             // x fragments straight from global memory need K to be a whole number of chunks (no bounds checks
             // in the kernel); otherwise x is staged in shared memory with zeros beyond K
             const bool direct = cfg.xdirect && (L.K % L.chunk_k) == 0;
-            const int x_bytes = direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
+            const int a8_span = ks_cta * cps * L.chunk_k;
+            const int x_bytes = a8 ? ((M * (a8_span + 16) + 15) / 16) * 16 + a8_span
+                                   : direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
             const double warps = (double)n_rb * ks;
@@ -574,6 +578,62 @@ extern "C" ql_status qlinear_forward_gated(qlinear_t hg, qlinear_t hu, const voi
     if (s != QL_OK) return s;
     const int blocks = (int)std::min<int64_t>((n + 255) / 256, (int64_t)hg->num_sms * 8);
     gate_mul_kernel<<<blocks, 256, 0, st>>>(g, u, static_cast<__half*>(y), n, act);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+namespace {
+template <int BITS, bool GROUPED>
+cudaError_t launch_a8(const qlinear_s* h, const GemvA8Params& prm, const GemvPlan& pl, cudaStream_t st)
+{
+    static std::atomic<bool> attr_set[kMaxDevices];
+    auto kern = gemv_a8_kernel<BITS, GROUPED>;
+    cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, kGemvMaxSmem);
+    if (e != cudaSuccess) return e;
+    return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
+}
+}  // namespace
+
+extern "C" ql_status qlinear_forward_a8(qlinear_t h, const void* x, void* y, int32_t M, void* stream)
+{
+    if (!h || !x || !y || M < 1) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
+    if (M > 8 || M > h->gemv_max_m) return QL_ERR_UNSUPPORTED;          // the decode stage only
+    if (device_timed_out(h)) return QL_ERR_DEVICE_TIMEOUT;
+    const Layout& L = h->L;
+    const GemvPlan pl = plan_gemv(L, h->n_rb, M, h->num_sms, false, true);
+    if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    GemvA8Params prm{};
+    prm.body = h->blob + L.body_offset;
+    prm.chan_scales = L.grouped ? nullptr : reinterpret_cast<const __half*>(h->blob + L.chan_scale_offset);
+    prm.x = static_cast<const __half*>(x);
+    prm.y = static_cast<__half*>(y);
+    prm.M = M; prm.N = L.N; prm.K = L.K;
+    prm.n_rb = h->n_rb; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
+    prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps;
+    const int span = pl.ks_cta * pl.cps * L.chunk_k;
+    prm.xq_stride = span + 16;
+    prm.xq_bytes = ((M * prm.xq_stride + 15) / 16) * 16;
+    prm.sg_bytes = span;                                                 // 32 bytes per 32-k group
+    cudaError_t e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (L.bits == 8) e = launch_a8<8, false>(h, prm, pl, st);
+    else if (L.grouped) e = launch_a8<4, true>(h, prm, pl, st);
+    else e = launch_a8<4, false>(h, prm, pl, st);
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_quantize_activations(const void* x, int8_t* xq, float* scale, int32_t M, int32_t K, int device, void* stream)
+{
+    if (!x || !xq || !scale || M < 1 || K < 32 || (K % 32)) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(xq)) & 15) return QL_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(scale) & 3) return QL_ERR_INVALID_ARG;
+    if (device < 0 || device >= kMaxDevices) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    quantize_activations_kernel<<<M, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __half*>(x),
+                                                                                reinterpret_cast<signed char*>(xq), scale, M, K);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 

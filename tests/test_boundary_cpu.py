@@ -21,7 +21,7 @@ def P(_built_library):
 def test_library_exports_every_declared_symbol(P):
     text = open(os.path.join(ROOT, "include", "qlinear.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    declared = sorted(set(re.findall(r"\b(qlinear_[a-z_]+)\s*\(", text)))
+    declared = sorted(set(re.findall(r"\b(qlinear_[a-z0-9_]+)\s*\(", text)))
     assert declared, "no declarations found"
     raw = ctypes.CDLL(P.LIB_PATH)
     for name in declared:
