@@ -33,7 +33,7 @@ struct GemvA8Params {
     int32_t M, N, K;
     int32_t n_rb, n_kc, block_bytes;
     int32_t ks_cta, ks_cta_log2, cl, cps;
-    int32_t xq_stride;                   // bytes between tokens in the shared xq slab (span + 16)
+    int32_t xq_stride;                   // bytes between tokens in the shared xq slab (span + 32: rows land 8 banks apart)
     int32_t xq_bytes;                    // bytes of the slab
     int32_t sg_bytes;                    // bytes of the per-group sums that follow it
 };
@@ -46,12 +46,20 @@ __device__ __forceinline__ void imma_16832(int d[4], const uint32_t a[4], uint32
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]));
 }
 
-// Step 1 for one value, bit for bit as stated above.
-__device__ __forceinline__ int quantize_one(float x, float r)
+// Step 1 for one value, bit for bit as stated above.  |x| <= amax gives |x * r| <= 127 (1 + 2^-22), which rounds
+// into [-127, 127] by itself: the clamp of the definition never acts, and is left to the byte packing's saturation.
+__device__ __forceinline__ int quantize_one(float x, float r) { return __float2int_rn(__fmul_rn(x, r)); }
+
+// Four s32 values in [-128, 127] as the four bytes of a word (lowest byte first).
+__device__ __forceinline__ uint32_t pack_s8x4(int b0, int b1, int b2, int b3)
 {
-    const int q = __float2int_rn(__fmul_rn(x, r));
-    return max(-127, min(127, q));
+    uint32_t hi, out;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi) : "r"(b3), "r"(b2));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(b1), "r"(b0), "r"(hi));
+    return out;
 }
+// Sum of the four signed bytes of a word.
+__device__ __forceinline__ int sum_s8x4(uint32_t w) { return __dp4a((int)w, 0x01010101, 0); }
 
 template <int BITS, bool GROUPED>
 __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Params p)
@@ -117,17 +125,26 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Pa
 #pragma unroll
         for (int m = 0; m < 8; ++m) am[m] = 0.f;
         const int vec_per_row = p.K >> 3;
+        // eight independent 16-byte loads per thread and turn, so that their latencies overlap
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
             if (m < p.M) {
                 const uint4* row = reinterpret_cast<const uint4*>(p.x + (int64_t)m * p.K);
-                for (int v = threadIdx.x; v < vec_per_row; v += kGemvThreads) {
-                    const uint4 u = row[v];
-                    const __half2* h = reinterpret_cast<const __half2*>(&u);
+                for (int v0 = threadIdx.x; v0 < vec_per_row; v0 += 8 * kGemvThreads) {
+                    uint4 u[8];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 f = __half22float2(h[j]);
-                        am[m] = fmaxf(am[m], fmaxf(fabsf(f.x), fabsf(f.y)));
+                    for (int j = 0; j < 8; ++j) {
+                        const int v = v0 + j * kGemvThreads;
+                        u[j] = v < vec_per_row ? row[v] : make_uint4(0, 0, 0, 0);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const __half2* h = reinterpret_cast<const __half2*>(&u[j]);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float2 f = __half22float2(__habs2(h[i]));
+                            am[m] = fmaxf(am[m], fmaxf(f.x, f.y));
+                        }
                     }
                 }
             }
@@ -151,38 +168,46 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Pa
     }
     // ---- step 1b: quantise this CTA's K range, and -OFFSET * (sum of xq) per token and 32-k group
     {
-        const int vec_per_tok = span >> 3, total = p.M * vec_per_tok;     // 8 values per thread and turn; 4 threads per group
-        for (int i0 = warp * 32; i0 < total; i0 += kGemvThreads) {
-            const int i = i0 + lane;
-            int q8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-            int m = 0, v = 0;
-            if (i < total) {
-                m = i / vec_per_tok;
-                v = i - m * vec_per_tok;
-                const int k = k_cta0 + v * 8;
-                if (k < p.K) {
-                    const uint4 u = *reinterpret_cast<const uint4*>(p.x + (int64_t)m * p.K + k);
-                    const __half2* h = reinterpret_cast<const __half2*>(&u);
-                    const float r = recip_x[m];
+        // 8 values per thread and turn, 4 threads per 32-k group; four turns' loads are issued together
+        const int vec_per_tok = span >> 3, total = p.M * vec_per_tok;
+        constexpr int B = 4;
+        for (int i0 = warp * 32; i0 < total; i0 += B * kGemvThreads) {
+            uint4 u[B];
+            int mm[B], vv[B];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float2 f = __half22float2(h[j]);
-                        q8[2 * j] = quantize_one(f.x, r);
-                        q8[2 * j + 1] = quantize_one(f.y, r);
-                    }
+            for (int b = 0; b < B; ++b) {
+                const int i = i0 + b * kGemvThreads + lane;
+                mm[b] = 0; vv[b] = 0;
+                u[b] = make_uint4(0, 0, 0, 0);
+                if (i < total) {
+                    mm[b] = i / vec_per_tok;
+                    vv[b] = i - mm[b] * vec_per_tok;
+                    const int k = k_cta0 + vv[b] * 8;
+                    if (k < p.K) u[b] = *reinterpret_cast<const uint4*>(p.x + (int64_t)mm[b] * p.K + k);
                 }
-                auto pack4 = [](int a, int b, int cc, int d) {
-                    return (uint32_t)(a & 0xFF) | ((uint32_t)(b & 0xFF) << 8) | ((uint32_t)(cc & 0xFF) << 16) | ((uint32_t)(d & 0xFF) << 24);
-                };
-                uint2 out;
-                if (BITS == 4) { out.x = pack4(q8[0], q8[2], q8[1], q8[3]); out.y = pack4(q8[4], q8[6], q8[5], q8[7]); }
-                else { out.x = pack4(q8[0], q8[1], q8[2], q8[3]); out.y = pack4(q8[4], q8[5], q8[6], q8[7]); }
-                *reinterpret_cast<uint2*>(xq + m * p.xq_stride + v * 8) = out;
             }
-            int s8 = q8[0] + q8[1] + q8[2] + q8[3] + q8[4] + q8[5] + q8[6] + q8[7];
-            s8 += __shfl_xor_sync(0xffffffffu, s8, 1);
-            s8 += __shfl_xor_sync(0xffffffffu, s8, 2);
-            if (i < total && (lane & 3) == 0) sg[(v >> 2) * 8 + m] = -OFFSET * s8;
+#pragma unroll
+            for (int b = 0; b < B; ++b) {
+                if (i0 + b * kGemvThreads >= total) break;               // (warp-uniform)
+                const int i = i0 + b * kGemvThreads + lane, m = mm[b], v = vv[b];
+                const __half2* h = reinterpret_cast<const __half2*>(&u[b]);
+                const float r = recip_x[m];
+                int q8[8];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float2 f = __half22float2(h[j]);
+                    q8[2 * j] = quantize_one(f.x, r);
+                    q8[2 * j + 1] = quantize_one(f.y, r);
+                }
+                uint2 out;
+                if (BITS == 4) { out.x = pack_s8x4(q8[0], q8[2], q8[1], q8[3]); out.y = pack_s8x4(q8[4], q8[6], q8[5], q8[7]); }
+                else { out.x = pack_s8x4(q8[0], q8[1], q8[2], q8[3]); out.y = pack_s8x4(q8[4], q8[5], q8[6], q8[7]); }
+                if (i < total) *reinterpret_cast<uint2*>(xq + m * p.xq_stride + v * 8) = out;
+                int s8 = sum_s8x4(out.x) + sum_s8x4(out.y);
+                s8 += __shfl_xor_sync(0xffffffffu, s8, 1);
+                s8 += __shfl_xor_sync(0xffffffffu, s8, 2);
+                if (i < total && (lane & 3) == 0) sg[(v >> 2) * 8 + m] = -OFFSET * s8;
+            }
         }
         __syncthreads();
     }
@@ -348,8 +373,8 @@ __global__ void __launch_bounds__(256) quantize_activations_kernel(const __half*
             q8[2 * j + 1] = quantize_one(f.y, r);
         }
         uint2 out;
-        out.x = (uint32_t)(q8[0] & 0xFF) | ((uint32_t)(q8[1] & 0xFF) << 8) | ((uint32_t)(q8[2] & 0xFF) << 16) | ((uint32_t)(q8[3] & 0xFF) << 24);
-        out.y = (uint32_t)(q8[4] & 0xFF) | ((uint32_t)(q8[5] & 0xFF) << 8) | ((uint32_t)(q8[6] & 0xFF) << 16) | ((uint32_t)(q8[7] & 0xFF) << 24);
+        out.x = pack_s8x4(q8[0], q8[1], q8[2], q8[3]);
+        out.y = pack_s8x4(q8[4], q8[5], q8[6], q8[7]);
         *reinterpret_cast<uint2*>(xq + (int64_t)m * K + v * 8) = out;
     }
 }

@@ -154,7 +154,7 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = f
             // in the kernel); otherwise x is staged in shared memory with zeros beyond K
             const bool direct = cfg.xdirect && (L.K % L.chunk_k) == 0;
             const int a8_span = ks_cta * cps * L.chunk_k;
-            const int x_bytes = a8 ? ((M * (a8_span + 16) + 15) / 16) * 16 + a8_span
+            const int x_bytes = a8 ? ((M * (a8_span + 32) + 15) / 16) * 16 + a8_span
                                    : direct ? 0 : ((M * x_stride * 2 + 127) / 128) * 128;
             const int smem = x_bytes + kGemvWarps * (kGemvRing * 512 + (L.grouped ? 1024 : 0));
             if (smem > kGemvMaxSmem) continue;
@@ -613,7 +613,7 @@ extern "C" ql_status qlinear_forward_a8(qlinear_t h, const void* x, void* y, int
     prm.n_rb = h->n_rb; prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps;
     const int span = pl.ks_cta * pl.cps * L.chunk_k;
-    prm.xq_stride = span + 16;
+    prm.xq_stride = span + 32;
     prm.xq_bytes = ((M * prm.xq_stride + 15) / 16) * 16;
     prm.sg_bytes = span;                                                 // 32 bytes per 32-k group
     cudaError_t e;
