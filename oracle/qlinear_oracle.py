@@ -212,6 +212,35 @@ def linear_int8_activations(x, q, s, group: int):
 # dimension for V), the reading recorded in the design notes: the paper does not say how its cache is stored.
 
 
+def kv_quantize_rows(a: np.ndarray):
+    """fp16 [T, d] -> (int8 [T, d], fp16 scale [T]): one scale per row (per cached token),
+    s = fp16(amax / 127) with the division in fp32, q = round-half-even(a / s) in fp32 clamped to [-127, 127];
+    a row whose scale rounds to zero (all zeros, or below fp16's range) is stored as zeros with scale 1."""
+    a32 = np.asarray(a, dtype=np.float16).astype(np.float32)
+    amax = np.abs(a32).max(axis=1)
+    s16 = (amax / np.float32(127.0)).astype(np.float32).astype(np.float16)
+    dead = s16.astype(np.float32) == 0
+    sf = np.where(dead, np.float32(1.0), s16.astype(np.float32)).astype(np.float32)
+    with np.errstate(over="ignore"):
+        v = (a32 / sf[:, None]).astype(np.float32)
+    q = np.clip(np.rint(v), -127, 127).astype(np.int8)
+    q[dead] = 0
+    return q, np.where(dead, np.float16(1.0), s16).astype(np.float16)
+
+
+def kv_attention(qry, k, v, prob):
+    """The two attention products over a cache built from fp16 keys k [T, d] and values v [T, d]:
+    returns (scores64 [R, T], A_scores, out64 [R, d], A_out).  The value scales are per token, i.e. per INPUT
+    channel of the V layer, so they are folded into the probabilities first: x' = fp16(prob * s_v) (the product of
+    two fp16 numbers is exact in fp32; one rounding to fp16), out = x' . q_v with unit channel scales."""
+    k_q, k_s = kv_quantize_rows(k)
+    v_q, v_s = kv_quantize_rows(v)
+    sc64, A_sc, _ = kv_scores(qry, k_q, k_s)
+    xp = (np.asarray(prob, np.float16).astype(np.float32) * v_s.astype(np.float32)[None, :]).astype(np.float16)
+    out64, A_out, _ = kv_output(xp, np.ascontiguousarray(v_q.T), np.ones(v_q.shape[1], np.float16))
+    return sc64, A_sc, out64, A_out
+
+
 def kv_scores(qry, k_q, k_s):
     """scores64 [R, T] = qry [R, d_h] . Kcache^T, K cache k_q int8 [T, d_h] (O = T, I = d_h), k_s fp16 [T]."""
     return linear(qry, k_q, k_s, 0)

@@ -184,3 +184,45 @@ def test_kv_products_against_plain_loops():
         for j in range(d):                                   # one output per head dimension: O = d_h, I = cache positions
             want = sum(float(prob[r, t]) * float(v_s[j]) * int(v_q[j, t]) for t in range(T))
             assert abs(out[r, j] - want) <= 1e-12 * max(1.0, abs(want))
+
+
+def test_kv_row_quantisation_hand_cases():
+    # row 0: amax = 127 / 64 exactly, so s = 1/64 and every quotient is exact; -0.5/64 * 64 = -0.5 is a tie (to even: -0)
+    # row 1: all zeros -> zeros with scale 1
+    # row 2: amax = 1: s = fp16(1/127) = 0.00787353515625 (rounded DOWN), 1 / s = 127.0078 -> 127
+    # row 3: a scale in fp16's subnormal range: 1.4 * 2^-24 rounds to 2^-24, the quotient 177.8 is clamped to 127
+    rows = np.zeros((4, 4), np.float64)
+    rows[0] = [127 / 64, -63.5 / 64, 0.5 / 64, 2.5 / 64]
+    rows[2] = [1.0, -0.5, 0.25, 0.004]
+    rows[3] = [127 * 1.4 * 2.0 ** -24, 2.0 ** -24, 0, 0]
+    a = rows.astype(np.float16)
+    q, s = O.kv_quantize_rows(a)
+    assert s[0] == np.float16(1 / 64) and q[0].tolist() == [127, -64, 0, 2]
+    assert s[1] == np.float16(1.0) and not q[1].any()
+    assert float(s[2]) == 0.00787353515625 and q[2].tolist() == [127, -64, 32, 1]
+    assert float(s[3]) == 2.0 ** -24 and q[3, 0] == 127 and q[3, 1] == 1
+    assert np.abs(q).max() <= 127
+
+
+def test_kv_attention_matches_a_plain_float_attention_closely_and_exactly_on_the_grid():
+    rng = np.random.default_rng(17)
+    T, d, R = 96, 32, 4
+    k = rng.standard_normal((T, d)).astype(np.float16)
+    v = rng.standard_normal((T, d)).astype(np.float16)
+    qry = rng.standard_normal((R, d)).astype(np.float16)
+    prob = rng.uniform(0, 1, size=(R, T)).astype(np.float16)
+    sc64, _, out64, _ = O.kv_attention(qry, k, v, prob)
+    sc_ref = qry.astype(np.float64) @ k.astype(np.float64).T
+    out_ref = prob.astype(np.float64) @ v.astype(np.float64)
+    assert np.linalg.norm(sc64 - sc_ref) / np.linalg.norm(sc_ref) < 1e-2          # int8 noise, nothing structural
+    assert np.linalg.norm(out64 - out_ref) / np.linalg.norm(out_ref) < 1e-2
+    # keys and values already on an int8 grid with power-of-two scales, probabilities that are powers of two:
+    # every step is exact, so the result equals plain fp64 attention
+    ki = rng.integers(-127, 128, size=(T, d)); ki[:, 0] = 127
+    vi = rng.integers(-127, 128, size=(T, d)); vi[:, 0] = -127
+    kg = (ki * 2.0 ** -5).astype(np.float16)
+    vg = (vi * 2.0 ** -6).astype(np.float16)
+    pg = (2.0 ** -rng.integers(1, 6, size=(R, T))).astype(np.float16)
+    sc64, _, out64, _ = O.kv_attention(qry, kg, vg, pg)
+    np.testing.assert_allclose(sc64, qry.astype(np.float64) @ kg.astype(np.float64).T, rtol=1e-13, atol=1e-12)
+    np.testing.assert_allclose(out64, pg.astype(np.float64) @ vg.astype(np.float64), rtol=1e-13, atol=1e-12)
