@@ -93,7 +93,8 @@ ql_status qlinear_unpack(const qlinear_desc* desc, const void* packed, int8_t* q
 /* Binds a packed blob that already lives in DEVICE memory to a handle (Section 3.4: the converted
  * weights stay resident in GPU memory and serve both stages, Section 3.7).
  *   packed_dev  device pointer, 256-byte aligned, qlinear_packed_size(desc) bytes, owned by the caller,
- *               must stay alive and unchanged until qlinear_destroy.
+ *               must stay alive and unchanged until qlinear_destroy (the KV-cache calls below are the one exception:
+ *               they write into their blobs).
  *   device      CUDA device ordinal that owns packed_dev.
  * The handle owns host memory only (shape, kernel plans); the first handle on a device also creates that
  * device's shared buffers (see "Device memory" above), so the first create on a device should come before
@@ -174,6 +175,35 @@ ql_status qlinear_forward_a8(qlinear_t h, const void* x_dev, void* y_dev, int32_
  * Errors: QL_ERR_INVALID_ARG, QL_ERR_CUDA. */
 ql_status qlinear_quantize_activations(const void* x_dev, int8_t* xq_dev, float* scale_dev, int32_t M, int32_t K,
                                        int device, void* cuda_stream);
+
+/* The KV cache held as weights (Section 3.8, "GPU-Optimized KV Cache Layout"): the K cache is a layer with
+ * O = cache positions and I = head dimension d_h (it stands for K^T in Q K^T), the V cache a layer with O = d_h and
+ * I = cache positions, so that both attention products are calls of the linear kernels and the second comes out as
+ * [query rows, d_h], the layout the paper's QKV transformation wants (rows = S * h_q / h_kv per KV head).
+ * The paper does not say how its cache is stored; here both caches are int8 blobs (Section 4.2's 8-bit format)
+ * with one scale per cached TOKEN:  s = fp16(max|v| / 127),  q = round-half-to-even(v / s) clamped to +-127, IEEE
+ * fp32 operations (a vector whose scale rounds to zero is stored as zeros with scale 1).
+ *
+ * A cache pair is two ordinary handles over caller-owned blobs that the caller packed from ZERO weights:
+ *   h_k  desc {N = cache positions, K = d_h, bits 8, group 0}, channel scales 0 (an empty position scores 0)
+ *   h_v  desc {N = d_h, K = cache positions, bits 8, group 0}, channel scales 1
+ * qlinear_kv_append quantises n_new key and value vectors (k_new_dev, v_new_dev: fp16 [n_new, d_h]) and writes them
+ * to positions pos .. pos + n_new - 1: the key integers and their scales into the K blob (a token is an output
+ * channel there), the value integers into the V blob and their scales into v_scale_dev (fp16 [cache positions],
+ * caller-owned): in the V cache a token is an INPUT channel, so its scale is folded into the probabilities instead,
+ *     out[r, d] = sum_t (prob[r, t] * s_v[t]) * q_v[t, d].
+ * These are the only calls that write to a blob; they must be ordered against forward calls on the same handles.
+ * qlinear_kv_scores:  scores_dev [R, cache positions] = q_rows_dev [R, d_h] . K^T   (= qlinear_forward on h_k).
+ * qlinear_kv_output:  out_dev [R, d_h] from prob_dev fp16 [R, cache positions]; tmp_dev is caller-owned scratch of
+ *                     the same shape as prob_dev (it receives prob * s_v rounded to fp16).
+ * Masking and the softmax between the two are the caller's.  Asynchronous, allocate nothing.
+ * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, handles that are not an int8 cache pair of matching
+ * shape, pos + n_new beyond the cache, d_h > 1024), otherwise as qlinear_forward. */
+ql_status qlinear_kv_append(qlinear_t h_k, qlinear_t h_v, const void* k_new_dev, const void* v_new_dev, void* v_scale_dev,
+                            int32_t pos, int32_t n_new, void* cuda_stream);
+ql_status qlinear_kv_scores(qlinear_t h_k, const void* q_rows_dev, void* scores_dev, int32_t R, void* cuda_stream);
+ql_status qlinear_kv_output(qlinear_t h_v, const void* prob_dev, const void* v_scale_dev, void* tmp_dev, void* out_dev,
+                            int32_t R, void* cuda_stream);
 
 /* Embedding lookup from a quantised table (Section 4.2: the mixed 8/4/4 scheme keeps the embedding table
  * in int4 like the feed-forward weights).  The handle's layer is read as a table of N rows of K values:

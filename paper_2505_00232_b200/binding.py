@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_embed",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -68,6 +68,12 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_forward_a8.restype = ctypes.c_int
     lib.qlinear_quantize_activations.argtypes = [vp, vp, vp, i32, i32, ctypes.c_int, vp]
     lib.qlinear_quantize_activations.restype = ctypes.c_int
+    lib.qlinear_kv_append.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
+    lib.qlinear_kv_append.restype = ctypes.c_int
+    lib.qlinear_kv_scores.argtypes = [vp, vp, vp, i32, vp]
+    lib.qlinear_kv_scores.restype = ctypes.c_int
+    lib.qlinear_kv_output.argtypes = [vp, vp, vp, vp, vp, i32, vp]
+    lib.qlinear_kv_output.restype = ctypes.c_int
     lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
     lib.qlinear_embed.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
@@ -333,3 +339,51 @@ class QLinear:
             self.close()
         except Exception:
             pass
+
+
+class KVCache:
+    """One KV head's cache held as two int8 weight blobs (see include/qlinear.h, qlinear_kv_append): argument
+    marshalling only -- the blobs start as the packed form of zero weights, every later byte is written by the library."""
+
+    def __init__(self, cache_size: int, d_h: int, device="cuda:0"):
+        import torch
+        self.cache_size, self.d_h, self.length = cache_size, d_h, 0
+        kd, vd = Desc(cache_size, d_h, 8, 0), Desc(d_h, cache_size, 8, 0)
+        self.k = QLinear(kd, qlinear_pack(kd, np.zeros((cache_size, d_h), np.int8), np.zeros((cache_size, 1), np.float16)), device)
+        self.v = QLinear(vd, qlinear_pack(vd, np.zeros((d_h, cache_size), np.int8), np.ones((d_h, 1), np.float16)), device)
+        self.v_scale = torch.zeros((cache_size,), dtype=torch.float16, device=device)
+
+    def append(self, k_new, v_new, stream=None):
+        """k_new, v_new: fp16 CUDA [n_new, d_h], written to positions length .. length + n_new - 1."""
+        import torch
+        for t in (k_new, v_new):
+            if t.dim() != 2 or t.shape[1] != self.d_h or t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous():
+                raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_append (k_new, v_new must be contiguous fp16 CUDA [n, d_h])")
+        n = k_new.shape[0]
+        if v_new.shape[0] != n:
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_append (k_new and v_new differ in length)")
+        _check(lib.qlinear_kv_append(self.k._h, self.v._h, ctypes.c_void_p(k_new.data_ptr()), ctypes.c_void_p(v_new.data_ptr()),
+                                     ctypes.c_void_p(self.v_scale.data_ptr()), self.length, n, _stream_ptr(stream)), "qlinear_kv_append")
+        self.length += n
+
+    def scores(self, q_rows, stream=None):
+        """q_rows fp16 [R, d_h] -> fp16 [R, cache_size] (positions beyond `length` score 0)."""
+        import torch
+        if q_rows.dim() != 2 or q_rows.shape[1] != self.d_h or q_rows.dtype != torch.float16 or not q_rows.is_cuda or not q_rows.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_scores (q_rows must be contiguous fp16 CUDA [R, d_h])")
+        out = torch.empty((q_rows.shape[0], self.cache_size), dtype=torch.float16, device=q_rows.device)
+        _check(lib.qlinear_kv_scores(self.k._h, ctypes.c_void_p(q_rows.data_ptr()), ctypes.c_void_p(out.data_ptr()), q_rows.shape[0],
+                                     _stream_ptr(stream)), "qlinear_kv_scores")
+        return out
+
+    def output(self, prob, stream=None):
+        """prob fp16 [R, cache_size] -> fp16 [R, d_h]."""
+        import torch
+        if prob.dim() != 2 or prob.shape[1] != self.cache_size or prob.dtype != torch.float16 or not prob.is_cuda or not prob.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_output (prob must be contiguous fp16 CUDA [R, cache_size])")
+        tmp = torch.empty_like(prob)
+        out = torch.empty((prob.shape[0], self.d_h), dtype=torch.float16, device=prob.device)
+        _check(lib.qlinear_kv_output(self.v._h, ctypes.c_void_p(prob.data_ptr()), ctypes.c_void_p(self.v_scale.data_ptr()),
+                                     ctypes.c_void_p(tmp.data_ptr()), ctypes.c_void_p(out.data_ptr()), prob.shape[0], _stream_ptr(stream)),
+               "qlinear_kv_output")
+        return out

@@ -27,6 +27,7 @@ __device__ unsigned int* g_status_host;
 #include "gemv.cuh"
 #include "gemv_stream.cuh"
 #include "gemv_a8.cuh"
+#include "kv.cuh"
 #include "gemm.cuh"
 #include "gemm_pair.cuh"
 
@@ -635,6 +636,56 @@ extern "C" ql_status qlinear_quantize_activations(const void* x, int8_t* xq, flo
     quantize_activations_kernel<<<M, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __half*>(x),
                                                                                 reinterpret_cast<signed char*>(xq), scale, M, K);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_kv_append(qlinear_t hk, qlinear_t hv, const void* k_new, const void* v_new, void* v_scale,
+                                       int32_t pos, int32_t n_new, void* stream)
+{
+    if (!hk || !hv || !k_new || !v_new || !v_scale || pos < 0 || n_new < 0) return QL_ERR_INVALID_ARG;
+    const Layout &K = hk->L, &V = hv->L;
+    if (hk->device != hv->device || K.bits != 8 || V.bits != 8 || K.N != V.K || K.K != V.N) return QL_ERR_INVALID_ARG;
+    if ((int64_t)pos + n_new > K.N || K.K > 1024) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(v_scale)) & 1) return QL_ERR_INVALID_ARG;
+    if (n_new == 0) return QL_OK;
+    DeviceGuard guard(hk->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    KvAppendParams prm{};
+    uint8_t* kb = const_cast<uint8_t*>(hk->blob);                        // the caches are the one kind of blob the library writes
+    uint8_t* vb = const_cast<uint8_t*>(hv->blob);
+    prm.k_body = kb + K.body_offset;
+    prm.k_scales = reinterpret_cast<__half*>(kb + K.chan_scale_offset);
+    prm.v_body = vb + V.body_offset;
+    prm.v_scale = static_cast<__half*>(v_scale);
+    prm.k_new = static_cast<const __half*>(k_new);
+    prm.v_new = static_cast<const __half*>(v_new);
+    prm.d_h = K.K; prm.cache_size = K.N; prm.pos = pos; prm.n_new = n_new;
+    prm.k_n_kc = K.n_kc; prm.v_n_kc = V.n_kc;
+    kv_append_kernel<<<n_new, 128, 0, static_cast<cudaStream_t>(stream)>>>(prm);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_kv_scores(qlinear_t hk, const void* q_rows, void* scores, int32_t R, void* stream)
+{
+    if (!hk || hk->L.bits != 8) return QL_ERR_INVALID_ARG;
+    return qlinear_forward(hk, q_rows, scores, R, stream);
+}
+
+extern "C" ql_status qlinear_kv_output(qlinear_t hv, const void* prob, const void* v_scale, void* tmp, void* out, int32_t R, void* stream)
+{
+    if (!hv || !prob || !v_scale || !tmp || !out || R < 1 || hv->L.bits != 8) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(tmp) | reinterpret_cast<uintptr_t>(out)) & 15) return QL_ERR_INVALID_ARG;
+    const int T = hv->L.K;
+    if ((int64_t)R * T > INT32_MAX) return QL_ERR_INVALID_ARG;
+    {
+        DeviceGuard guard(hv->device);
+        if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+        const int64_t n = (int64_t)R * T;
+        const int blocks = (int)std::min<int64_t>((n + 255) / 256, (int64_t)hv->num_sms * 8);
+        kv_scale_probs_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __half*>(prob),
+                                                                                     static_cast<const __half*>(v_scale), static_cast<__half*>(tmp), n, T);
+        if (cudaGetLastError() != cudaSuccess) return QL_ERR_CUDA;
+    }
+    return qlinear_forward(hv, tmp, out, R, stream);
 }
 
 extern "C" ql_status qlinear_embed(qlinear_t h, const int32_t* ids, int32_t n, void* y, void* stream)

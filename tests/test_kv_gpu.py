@@ -1,0 +1,90 @@
+"""The KV cache held as weights (paper Section 3.8) against the CPU oracle, through the C-ABI, on a B200: the
+protocol of the paper's LLM benchmark, 1024 prefill tokens then 256 decode steps (Section 4.2), for one KV head of
+a grouped-query model (4 query heads per KV head, d_h = 128)."""
+import numpy as np
+import pytest
+
+from oracle import qlinear_oracle as O
+from workloads import generators as gen
+
+pytestmark = pytest.mark.gpu
+
+CACHE, DH, GROUP = 1280, 128, 4
+
+
+@pytest.fixture(scope="module")
+def P(_built_library):
+    import paper_2505_00232_b200 as P
+    return P
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return torch
+
+
+def tensors(seed, T):
+    k = gen.normal_fp16(seed, 1, (T, DH))
+    v = gen.normal_fp16(seed, 2, (T, DH))
+    v[5, :] = 0                                         # a zero vector: stored as zeros with scale 1
+    k[7, :] *= np.float16(40.0)                         # per-token scales really differ
+    return k, v
+
+
+def test_append_writes_exactly_the_oracles_integers_and_scales(P, torch):
+    k, v = tensors(811, CACHE)
+    cache = P.KVCache(CACHE, DH)
+    kd, vd = torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda()
+    cache.append(kd[:1024], vd[:1024])                  # prefill: 1024 tokens in one call
+    for t in range(1024, CACHE):                        # decode: one token per step
+        cache.append(kd[t:t + 1], vd[t:t + 1])
+    torch.cuda.synchronize()
+    assert cache.length == CACHE and cache.k.device_status() == (0, 0)
+    k_q, k_s = O.kv_quantize_rows(k)
+    v_q, v_s = O.kv_quantize_rows(v)
+    assert (cache.k.debug_unpack().cpu().numpy() == k_q).all()           # K cache: O = positions, I = d_h
+    assert (cache.v.debug_unpack().cpu().numpy() == v_q.T).all()         # V cache: O = d_h, I = positions
+    _, ks_blob = P.qlinear_unpack(cache.k.desc, cache.k.packed.cpu().numpy())
+    assert (ks_blob.reshape(-1).view(np.uint16) == k_s.view(np.uint16)).all()
+    assert (cache.v_scale.cpu().numpy().view(np.uint16) == v_s.view(np.uint16)).all()
+
+
+@pytest.mark.parametrize("R,T", [(GROUP, 1280), (GROUP, 1031), (1, 200), (GROUP * 128, 1024)],
+                         ids=["decode-full-cache", "decode-partial-cache", "one-row", "prefill-512-rows"])
+def test_attention_products_match_the_oracle(P, torch, R, T):
+    """scores = Q K^T and out = P V through the linear kernels (R = S * h_q / h_kv query rows of one KV head),
+    inside the linear layer's tolerance; positions beyond the cache length score exactly 0."""
+    k, v = tensors(900 + T, T)
+    qry = gen.normal_fp16(900 + T, 3, (R, DH))
+    cache = P.KVCache(CACHE, DH)
+    cache.append(torch.from_numpy(k).cuda(), torch.from_numpy(v).cuda())
+    sc = cache.scores(torch.from_numpy(qry).cuda())
+    torch.cuda.synchronize()
+    sc_np = sc.cpu().numpy()
+    assert (sc_np[:, T:] == 0).all()
+    # probabilities: a softmax over the live positions (computed here in fp64: masking and softmax are the caller's)
+    z = sc_np[:, :T].astype(np.float64) / np.sqrt(DH)
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    prob = np.zeros((R, CACHE), np.float16)
+    prob[:, :T] = (p / p.sum(axis=1, keepdims=True)).astype(np.float16)
+    out = cache.output(torch.from_numpy(prob).cuda())
+    torch.cuda.synchronize()
+    sc64, A_sc, out64, A_out = O.kv_attention(qry, k, v, prob[:, :T])
+    ok, rel, worst = O.check_against(sc_np[:, :T], sc64, A_sc)
+    assert ok, ("scores", rel, worst)
+    ok, rel, worst = O.check_against(out.cpu().numpy(), out64, A_out)
+    assert ok, ("output", rel, worst)
+
+
+def test_append_argument_errors(P, torch):
+    cache = P.KVCache(256, 64)
+    a = torch.zeros((200, 64), dtype=torch.float16, device="cuda")
+    cache.append(a, a)
+    with pytest.raises(P.QLinearError):
+        cache.append(a, a)                              # 400 > 256 positions
+    other = P.KVCache(256, 32)
+    import ctypes
+    vp = ctypes.c_void_p
+    assert P.lib.qlinear_kv_append(cache.k._h, other.v._h, vp(a.data_ptr()), vp(a.data_ptr()), vp(cache.v_scale.data_ptr()), 0, 1, None) == 1
