@@ -218,6 +218,29 @@ class LayerSet:
         self.y_host_all.copy_(self.y_all, non_blocking=True)
         self.torch.cuda.current_stream().synchronize()
 
+    def e2e_graphs(self, grouped=False):
+        """The same end-to-end step captured once per weight copy as a CUDA graph (copy in, forwards, copy out):
+        what a serving loop that replays a fixed step does.  Returns one replay-and-synchronise callable per copy."""
+        torch = self.torch
+        graphs = []
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for cp in range(self.copies):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    self.x_all.copy_(self.x_host_all, non_blocking=True)
+                    (self.step_grouped if grouped else self.step)(cp)
+                    self.y_host_all.copy_(self.y_all, non_blocking=True)
+                graphs.append(g)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+
+        def run(cp):
+            graphs[cp].replay()
+            torch.cuda.current_stream().synchronize()
+        return run
+
     @property
     def h2d_bytes(self):
         return 2 * self.x_host_all.numel()
@@ -544,16 +567,21 @@ def main():
 
     # ---- end to end through the public API with host buffers: per step ONE H2D copy of all inputs from pinned
     # memory, the forwards, ONE D2H copy of all outputs, synchronise
-    for i in range(3):
-        ls.step_e2e(i % copies, grouped)
-    torch.cuda.synchronize()
-    e2e_steps, e2e_s = 0, 0.0
-    t0 = time.perf_counter()
-    while e2e_s < MIN_REGION_S / 2 or e2e_steps < 8:
-        ls.step_e2e(e2e_steps % copies, grouped)
-        e2e_steps += 1
-        e2e_s = time.perf_counter() - t0
-    e2e_s = max_over_ranks(e2e_s, device)
+    def time_e2e(step):
+        for i in range(3):
+            step(i % copies)
+        torch.cuda.synchronize()
+        n, dt = 0, 0.0
+        t0 = time.perf_counter()
+        while dt < MIN_REGION_S / 2 or n < 8:
+            step(n % copies)
+            n += 1
+            dt = time.perf_counter() - t0
+        return n, max_over_ranks(dt, device)
+    # plain calls (every step issues its copies and launches), and the same step replayed as one CUDA graph
+    e2e_steps_plain, e2e_s_plain = time_e2e(lambda cp: ls.step_e2e(cp, grouped))
+    e2e_plain = whole_job_value(units_per_step, e2e_steps_plain, e2e_s_plain * 1e3, world)
+    e2e_steps, e2e_s = time_e2e(ls.e2e_graphs(grouped)) if stage == "decode" else (e2e_steps_plain, e2e_s_plain)
     e2e_value = whole_job_value(units_per_step, e2e_steps, e2e_s * 1e3, world)
 
     # ---- roofline of the dominant kernel (live CUDA-event timing of that kernel's launches alone)
@@ -577,7 +605,10 @@ def main():
                    "parallelism": "replicas only" if world > 1 else "single gpu"},
         "clocks": res["clocks"], "gpu_launches": res["launches"],
         "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": ls.h2d_bytes, "d2h_bytes_per_step": ls.d2h_bytes,
-                "steps": e2e_steps, "copies": "one pinned host buffer each way: 1 H2D + 1 D2H per step"},
+                "steps": e2e_steps, "us_per_step": e2e_s / e2e_steps * 1e6,
+                "copies": "one pinned host buffer each way: 1 H2D + 1 D2H per step, host synchronises after every step",
+                "launch": "the step (copy in, forwards, copy out) replayed as one CUDA graph" if stage == "decode" else "stream launches",
+                "plain_calls": {"value": e2e_plain, "us_per_step": e2e_s_plain / e2e_steps_plain * 1e6, "steps": e2e_steps_plain}},
         "roofline": roof,
         "frac_of_measured_peak": value / world / (peaks["hbm_gbs"] if stage == "decode" else peaks["bf16_tflops"]),
     }
