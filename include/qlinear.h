@@ -163,8 +163,15 @@ ql_status qlinear_forward_gated(qlinear_t h_gate, qlinear_t h_up, const void* x_
  *     y[m,n] = fp16( (amax / 127) * sum_g s[n,g] * sum_{k in g} xq[m,k] * q[n,k] )
  * with the inner sums exact (integer tensor-core instructions).  The paper gives neither the granularity of the
  * activation scale nor the rounding; one scale per token, symmetric, is the reading taken here.
- *   h, x_dev, y_dev, cuda_stream as in qlinear_forward;  1 <= M <= 8 (QL_ERR_UNSUPPORTED beyond: the prefill
- *   form -- qlinear_quantize_activations followed by an integer matmul -- has only its first kernel so far).
+ *   h, x_dev, y_dev, cuda_stream as in qlinear_forward.
+ * M <= 8, every scheme: one decode launch with the quantisation inside it.
+ * M > 128, the paper's own per-channel schemes (group 0: q8 and per-channel int4), K a multiple of 128 and a
+ * multiple of 256 output channels after padding to 128: the prefill form of the same section -- the quantisation
+ * kernel (qlinear_quantize_activations, into the device's shared scratch), then the CTA-pair prefill kernel in its
+ * integer form: the stored weight integers go to the tensor cores unconverted (tcgen05.mma kind::i8, u8 x s8 -> s32
+ * in tensor memory), and the epilogue removes the storage offset and applies both scales.  Such calls use the shared
+ * scratch and must be ordered against each other and against K-split prefill calls.
+ * Anything else (grouped scales with M > 8, 9 <= M <= 128, other shapes): QL_ERR_UNSUPPORTED.
  * Asynchronous, allocates nothing.  The result differs from qlinear_forward's by the quantisation noise of x
  * (about 1 % relative for Gaussian x); it equals it to fp32 round-off when x already lies on the int8 grid. */
 ql_status qlinear_forward_a8(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);

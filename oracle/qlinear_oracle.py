@@ -195,7 +195,10 @@ def linear_int8_activations(x, q, s, group: int):
     G = K if group == 0 else group
     xq, scale_x = quantize_activations(x)
     M = xq.shape[0]
-    acc = np.einsum("mgk,ngk->mng", xq.astype(np.int64).reshape(M, K // G, G), q.astype(np.int64).reshape(N, K // G, G))
+    # exact integers through the fp64 matmul: every product is below 2^14 and a sum over K <= 2^24 terms stays far
+    # below 2^53, so fp64 represents every partial sum exactly whatever the summation order
+    xg, qg = xq.astype(np.float64).reshape(M, K // G, G), q.astype(np.float64).reshape(N, K // G, G)
+    acc = np.rint(np.stack([xg[:, g, :] @ qg[:, g, :].T for g in range(K // G)], axis=2)).astype(np.int64)
     s64 = np.asarray(s, dtype=np.float16).reshape(N, K // G).astype(np.float64)
     y64 = scale_x.astype(np.float64)[:, None] * np.einsum("mng,ng->mn", acc.astype(np.float64), s64)
     with np.errstate(over="ignore"):

@@ -61,6 +61,10 @@ struct GemmParams {
     int32_t rsb_end[4];
     int32_t n_layers;
     int32_t act;                             // pair kernel, gated form: activation of the gate branch (QL_ACT_*)
+    // pair kernel, integer form (x_map then describes the int8 activations): per-token scale and sum of the
+    // quantised row (device arrays, padded to whole token tiles)
+    const float* a8_scale;
+    const int32_t* a8_rowsum;
 };
 constexpr int kGemmMaxGroup = 4;
 
@@ -109,6 +113,45 @@ struct DequantLane {
         }
         *reinterpret_cast<uint4*>(at + off_lo) = lo;
         *reinterpret_cast<uint4*>(at + off_hi) = hi;
+    }
+};
+
+// The integer form's counterpart (paper Section 3.7: pre-quantised weights meet int8 activations in integer
+// instructions): the stored weight integers, as they are (q + 8 or q + 128, unsigned), become the K-major
+// 128-byte-swizzled u8 tile of a 128-k step.  Warp dw handles row-block (dw & 7) and half of the step's chunks.
+struct RepackLane {
+    int rbk, half, g, c, lane;
+    __device__ RepackLane(int dw, int lane_) : rbk(dw & 7), half(dw >> 3), g(lane_ >> 2), c(lane_ & 3), lane(lane_) {}
+    // 8 bytes (k0 .. k0 + 7, k0 a multiple of 8) of tile row r
+    __device__ __forceinline__ static void store8(unsigned char* at, int r, int k0, uint32_t lo, uint32_t hi)
+    {
+        *reinterpret_cast<uint2*>(at + r * 128 + ((((k0 >> 4) ^ (r & 7)) << 4) | (k0 & 8))) = make_uint2(lo, hi);
+    }
+    template <int BITS>
+    __device__ __forceinline__ void step(const unsigned char* wp, unsigned char* at) const
+    {
+        const int r0 = rbk * kRbRows + g;                                // rows r0 and r0 + 8
+        if (BITS == 8) {                                                 // 4 chunks of 32 k per step, two per warp
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int ch = 2 * half + j;
+                const uint4 w = *reinterpret_cast<const uint4*>(wp + ch * kWeightBlockBytes + rbk * 512 + lane * 16);
+                const int k0 = 32 * ch + 8 * c;
+                store8(at, r0, k0, __byte_perm(w.x, w.y, 0x5410), __byte_perm(w.z, w.w, 0x5410));
+                store8(at, r0 + 8, k0, __byte_perm(w.x, w.y, 0x7632), __byte_perm(w.z, w.w, 0x7632));
+            }
+        } else {                                                         // 2 chunks of 64 k per step, one per warp
+            const uint4 w = *reinterpret_cast<const uint4*>(wp + half * kWeightBlockBytes + rbk * 512 + lane * 16);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {                                // the chunk's two 32-k halves
+                // low nibbles of a word: row g at slots 0, 2, 1, 3; high nibbles: row g + 8 (layout.h)
+                const uint32_t a = ww[2 * h], b = ww[2 * h + 1];
+                const int k0 = 64 * half + 32 * h + 8 * c;
+                store8(at, r0, k0, __byte_perm(a & 0x0F0F0F0Fu, 0, 0x3120), __byte_perm(b & 0x0F0F0F0Fu, 0, 0x3120));
+                store8(at, r0 + 8, k0, __byte_perm((a >> 4) & 0x0F0F0F0Fu, 0, 0x3120), __byte_perm((b >> 4) & 0x0F0F0F0Fu, 0, 0x3120));
+            }
+        }
     }
 };
 
@@ -335,24 +378,25 @@ inline EncodeTiledFn get_encode_tiled()
 
 // The tensor map of x depends only on (pointer, K, M, box rows); callers reuse a few activation buffers, so the
 // last encodings are kept (per process, a handful of entries) instead of calling the driver on every forward.
-inline bool x_tensor_map(const void* x, int K, int M, int box_rows, CUtensorMap* out)
+// elem_bytes: 2 = fp16 activations (box 64 k wide), 1 = int8 activations (box 128 k wide); either way 128 bytes.
+inline bool x_tensor_map(const void* x, int K, int M, int box_rows, CUtensorMap* out, int elem_bytes = 2)
 {
-    struct Entry { const void* x; int K, M, rows; CUtensorMap map; };
+    struct Entry { const void* x; int K, M, rows, eb; CUtensorMap map; };
     constexpr int kEntries = 16;
     static Entry cache[kEntries] = {};
     static int next = 0;
     static std::mutex mu;
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < kEntries; ++i)
-        if (cache[i].x == x && cache[i].K == K && cache[i].M == M && cache[i].rows == box_rows) { *out = cache[i].map; return true; }
+        if (cache[i].x == x && cache[i].K == K && cache[i].M == M && cache[i].rows == box_rows && cache[i].eb == elem_bytes) { *out = cache[i].map; return true; }
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return false;
     const cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    const cuuint64_t gstr[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kGemmKStep, (cuuint32_t)box_rows};
+    const cuuint64_t gstr[1] = {(cuuint64_t)K * elem_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    Entry e{x, K, M, box_rows, {}};
-    if (enc(&e.map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
+    Entry e{x, K, M, box_rows, elem_bytes, {}};
+    if (enc(&e.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(x), gdim, gstr, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;

@@ -26,14 +26,16 @@ constexpr int kPairThreads = 28 * 32;
 // TB = token blocks (of 256) per tile.  With TB = 2 every dequantised A slot feeds two MMA groups (two
 // accumulators of 256 columns fill the tensor memory, so the epilogue is no longer hidden under the next
 // tile): half the dequantise work and half the A-slot hand-offs per flop.
-template <int BITS, int TB>
+// I8: the integer form (int8 activations, kind::i8): a k-step is 128 k, i.e. again 128 bytes per tile row.
+template <int BITS, int TB, bool I8 = false>
 struct GemmPairSmem {
-    static constexpr int kXBlockBytes = 128 * 128;                       // this CTA's 128 tokens x 64 k of one token block
+    static constexpr int kKStep = I8 ? 128 : kGemmKStep;
+    static constexpr int kXBlockBytes = 128 * 128;                       // this CTA's 128 tokens x one k-step of one token block
     static constexpr int kXBytes = TB * kXBlockBytes;
-    static constexpr int kWpkStride = BITS == 4 ? 5120 : 8192;           // packed block(s) of one k-step
+    static constexpr int kWpkStride = I8 ? (BITS == 4 ? 8192 : 16384) : (BITS == 4 ? 5120 : 8192);   // packed block(s) of one k-step
     static constexpr int kStageBytes = kXBytes + kWpkStride;
-    static constexpr int kStages = TB == 2 ? 4 : (BITS == 4 ? 6 : 5);
-    static constexpr int kASlots = TB == 2 ? 4 : 5;                      // one relay warp per slot (spare warps 5, 9, 13, 17, 21)
+    static constexpr int kStages = I8 ? (BITS == 4 ? 6 : 4) : TB == 2 ? 4 : (BITS == 4 ? 6 : 5);
+    static constexpr int kASlots = (I8 || TB == 2) ? 4 : 5;              // one relay warp per slot (spare warps 5, 9, 13, 17, 21)
     static constexpr int kAOffset = kStages * kStageBytes;
     static constexpr int kBarOffset = kAOffset + kASlots * kGemmATileBytes;
     static constexpr int kTotal = kBarOffset + 512 + 1024;               // barriers + alignment slack
@@ -78,12 +80,16 @@ __device__ __forceinline__ int pair_layer(const GemmParams& p, int& rsb)
 // place (tensor memory load, activation, tensor memory store); when the up tile is complete they write
 // fp16(act(gate) * up), the only tensor that ever goes to memory (paper Section 3.6), and free both accumulators.
 // Work unit t then counts (row super-block pair, token block) positions of ONE layer; every unit is two tiles.
-template <int BITS, bool GROUPED, int TB, bool GATED = false>
+// I8 (TB == 1, per-channel schemes, not gated): x_map describes int8 activations; the weight integers go to the A
+// tile unconverted (RepackLane), the MMAs are kind::i8 with an s32 accumulator, and the epilogue removes the storage
+// offset (off * sum of the token's quantised row) and applies both scales (paper Section 3.7, prefill stage).
+template <int BITS, bool GROUPED, int TB, bool GATED = false, bool I8 = false>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 {
     static_assert(!GATED || TB == 1, "the gated form uses both accumulators for one output tile");
-    using S = GemmPairSmem<BITS, TB>;
+    static_assert(!I8 || (TB == 1 && !GATED && !GROUPED), "the integer form: per-channel scales, 256-token tiles");
+    using S = GemmPairSmem<BITS, TB, I8>;
     constexpr int NS = S::kStages;
     constexpr int NA = S::kASlots;
     constexpr int BN = 256;                                              // tokens per MMA (128 per CTA)
@@ -148,7 +154,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         // ------------------------------------------------------------------ producer (each CTA feeds itself)
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
-            constexpr int CHUNKS = BITS == 4 ? 1 : 2;
+            constexpr int CHUNKS = S::kKStep / (BITS == 4 ? 64 : 32);      // packed blocks per k-step
             int s = 0, issued = 0;
             uint32_t par = 1;
             bool waited_dep = false, ok = true;
@@ -175,7 +181,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     }
 #pragma unroll
                     for (int tb = 0; tb < TB; ++tb)
-                        tma_load_2d(xs_addr(s) + tb * S::kXBlockBytes, &x_map, (step0 + it) * kGemmKStep, m0 + tb * BN, full_bar(s));
+                        tma_load_2d(xs_addr(s) + tb * S::kXBlockBytes, &x_map, (step0 + it) * S::kKStep, m0 + tb * BN, full_bar(s));
                     ++issued;
                     if (++s == NS) { s = 0; par ^= 1; }
                 }
@@ -188,7 +194,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            // f16 x f16 -> f32, or (integer form) u8 weights x s8 activations -> s32; both operands K-major, M = 256 per pair
+            constexpr uint32_t idesc = (I8 ? (2u << 4) | (1u << 10) : (1u << 4)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
             const uint32_t a_lo0 = umma_desc_lo(a_addr(0)), b_lo0 = umma_desc_lo(xs_addr(0));
             int s = 0, a = 0;
             uint32_t apar = 0;
@@ -212,10 +219,13 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 #pragma unroll
                     for (int tb = 0; tb < TB; ++tb) {
                         const uint32_t d = tmem_d + (uint32_t)(tb * BN), bl = b_lo + (uint32_t)tb * (S::kXBlockBytes >> 4);
-                        umma_f16_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
+                        if (I8) umma_i8_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
+                        else umma_f16_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k4 = 1; k4 < kGemmKStep / 16; ++k4)
-                            umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                        for (int k4 = 1; k4 < 4; ++k4) {                 // +32 bytes along K inside the swizzle row
+                            if (I8) umma_i8_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                            else umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                        }
                     }
                     umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
                     if (++s == NS) s = 0;
@@ -246,6 +256,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
             }
         } else {                                                         // 16 dequantise warps
         const DequantLane dq(warp - 2 - ((warp - 1) >> 2), lane);
+        const RepackLane rp(warp - 2 - ((warp - 1) >> 2), lane);
         int s = 0, a = 0;
         uint32_t par = 0;
         // A slot a was last read by the MMAs of step (gstep - NA); their retirement is the phase of the
@@ -263,7 +274,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                     if (!mbar_wait(empty_bar(s_old), par_old, abort_flag, 0xB00 + s_old)) { ok = false; break; }
                     if (++s_old == NS) { s_old = 0; par_old ^= 1; }
                 }
-                dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(a));
+                if (I8) rp.template step<BITS>(wpk_ptr(s), a_ptr(a));
+                else dq.template step<BITS, GROUPED>(wpk_ptr(s), a_ptr(a));
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(afull_bar(a));
@@ -324,6 +336,32 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive_remote(tempty_bar(0), 0); mbar_arrive_remote(tempty_bar(1), 0); }
+                continue;
+            }
+            if (I8) {
+                // acc = sum (q + off) * xq: remove off * (sum of the token's quantised row), then both scales
+                constexpr int OFF = BITS == 4 ? 8 : 128;
+                const float sn = n < N ? __half2float(p.lscales[ly][n]) : 0.f;
+                const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN);
+                __half* yr = p.ly[ly] + (int64_t)m0 * N + n;
+                const int ml = min(TILE_N, p.M - m0);
+#pragma unroll 1
+                for (int cc = 0; cc < ml; cc += 16) {
+                    uint32_t r[16];
+                    tmem_ld16(ta + (uint32_t)cc, r);
+                    if (n < N) {
+#pragma unroll
+                        for (int q = 0; q < 16; ++q)
+                            if (cc + q < ml) {
+                                const int tok = m0 + cc + q;
+                                const float v = (float)((int)r[q] - OFF * p.a8_rowsum[tok]);
+                                yr[(int64_t)(cc + q) * N] = __float2half_rn(p.a8_scale[tok] * (sn * v));
+                            }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(tempty_bar(buf), 0);
                 continue;
             }
             float scale = 1.f;
@@ -428,7 +466,9 @@ inline int gemm_pair_split(int tiles /* of the last, partial round */, int n_kst
     while (split > 1 && (n_ksteps % split || n_ksteps / split < 8 || tiles * split > clusters)) split >>= 1;
     return split == 3 ? 2 : split;                                       // the kernel adds 2 or 4 parts
 }
-inline size_t gemm_pair_scratch_bytes(int num_sms) { return (size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float); }
+// (at least 40 MB: the same buffer holds the int8 activations of the integer form, up to M x K = 2048 x 14336, and
+// the two projections of the unfused gating route)
+inline size_t gemm_pair_scratch_bytes(int num_sms) { return std::max<size_t>((size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float), (size_t)40 << 20); }
 inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 8; }
 
 // The layers of one launch: all read the same x and agree in K and scheme; each has an even number of row
@@ -442,15 +482,17 @@ struct GemmPairLayers {
 };
 
 // act < 0: the plain form.  act >= 0 (TB == 1): the gated form, set = {gate, up} of equal shape, y[0] the output.
-template <int BITS, bool GROUPED, int TB, bool GATED = false>
+// a8_scale != nullptr: the integer form; x is then the int8 activations, a8_scale / a8_rowsum their per-token arrays.
+template <int BITS, bool GROUPED, int TB, bool GATED = false, bool I8 = false>
 ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device,
-                           bool pdl, int num_sms, float* scratch, unsigned int* counters, int act = -1)
+                           bool pdl, int num_sms, float* scratch, unsigned int* counters, int act = -1,
+                           const float* a8_scale = nullptr, const int32_t* a8_rowsum = nullptr)
 {
-    using S = GemmPairSmem<BITS, TB>;
+    using S = GemmPairSmem<BITS, TB, I8>;
     const Layout& L = *set.L[0];
     CUtensorMap map;
-    if (!x_tensor_map(x, L.K, M, 128, &map)) return QL_ERR_CUDA;
-    auto kern = gemm_pair_kernel<BITS, GROUPED, TB, GATED>;
+    if (!x_tensor_map(x, L.K, M, 128, &map, I8 ? 1 : 2)) return QL_ERR_CUDA;
+    auto kern = gemm_pair_kernel<BITS, GROUPED, TB, GATED, I8>;
     static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
@@ -475,7 +517,8 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
     if (GATED) n_rsb = L.n_rsb;                                          // work units count positions of one layer
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
-    prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
+    prm.n_ksteps = (L.K + S::kKStep - 1) / S::kKStep;
+    prm.a8_scale = a8_scale; prm.a8_rowsum = a8_rowsum;
     prm.n_rsb = n_rsb;
     const int tiles = (n_rsb / 2) * ((M + 256 * TB - 1) / (256 * TB));
     // whole tiles fill the full rounds of the persistent grid; the tiles of the last partial round are split
@@ -483,7 +526,7 @@ ql_status gemm_pair_launch(const GemmPairLayers& set, const void* x, int M, cuda
     // (splitting the tail of a multi-round schedule was measured and does not pay: the exposed scratch
     // reduction costs what the shorter last round saves; only single-round layers are split)
     const int tail = tiles < clusters ? tiles : 0;
-    prm.split = (TB == 1 && !GATED) ? gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr) : 1;
+    prm.split = (TB == 1 && !GATED && !I8) ? gemm_pair_split(tail, prm.n_ksteps, num_sms, scratch != nullptr) : 1;
     prm.n_whole = prm.split > 1 ? tiles - tail : tiles;
     prm.scratch = scratch;
     prm.counters = counters;
@@ -539,6 +582,15 @@ inline ql_status gemm_pair_forward(const GemmPairLayers& set, const void* x, int
     if (L.bits == 8) return gemm_pair_launch<8, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
     if (L.grouped) return gemm_pair_launch<4, true, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
     return gemm_pair_launch<4, false, 1>(set, x, M, st, device, pdl, num_sms, scratch, counters);
+}
+
+// Integer form (per-channel schemes, K a multiple of 128): xq int8 [M, K] with per-token scale and row sum.
+inline ql_status gemm_pair_forward_i8(const GemmPairLayers& set, const void* xq, const float* scale, const int32_t* rowsum, int M,
+                                      cudaStream_t st, int device, bool pdl, int num_sms)
+{
+    const Layout& L = *set.L[0];
+    if (L.bits == 8) return gemm_pair_launch<8, false, 1, false, true>(set, xq, M, st, device, pdl, num_sms, nullptr, nullptr, -1, scale, rowsum);
+    return gemm_pair_launch<4, false, 1, false, true>(set, xq, M, st, device, pdl, num_sms, nullptr, nullptr, -1, scale, rowsum);
 }
 
 // Gated form: set = {gate, up}, both pair-applicable and of equal shape; y[0] receives act(gate) * up.

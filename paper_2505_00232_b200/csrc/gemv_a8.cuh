@@ -330,10 +330,12 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Pa
 }
 
 // The quantisation kernel of the prefill stage (Section 3.7): x fp16 [M, K] -> xq int8 [M, K] and one fp32
-// scale per token, by the same steps as above.  One CTA per token.
-__global__ void __launch_bounds__(256) quantize_activations_kernel(const __half* x, signed char* xq, float* scale, int M, int K)
+// scale per token, by the same steps as above; rowsum (may be null) receives the sum of each quantised row, which
+// the integer matmul needs to remove the weights' storage offset.  One CTA per token.
+__global__ void __launch_bounds__(256) quantize_activations_kernel(const __half* x, signed char* xq, float* scale, int32_t* rowsum, int M, int K)
 {
     __shared__ float wmax[8];
+    __shared__ int wsum[8];
     __shared__ float recip;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int m = blockIdx.x;
@@ -362,6 +364,7 @@ __global__ void __launch_bounds__(256) quantize_activations_kernel(const __half*
     }
     __syncthreads();
     const float r = recip;
+    int total = 0;
     for (int v = threadIdx.x; v < (K >> 3); v += 256) {
         const uint4 u = row[v];
         const __half2* h = reinterpret_cast<const __half2*>(&u);
@@ -376,6 +379,18 @@ __global__ void __launch_bounds__(256) quantize_activations_kernel(const __half*
         out.x = pack_s8x4(q8[0], q8[1], q8[2], q8[3]);
         out.y = pack_s8x4(q8[4], q8[5], q8[6], q8[7]);
         *reinterpret_cast<uint2*>(xq + (int64_t)m * K + v * 8) = out;
+        total += sum_s8x4(out.x) + sum_s8x4(out.y);
+    }
+    if (rowsum) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+        if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = total;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+            for (int w = 0; w < 8; ++w) t += wsum[w];
+            rowsum[m] = t;
+        }
     }
 }
 

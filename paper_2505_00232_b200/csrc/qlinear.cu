@@ -598,9 +598,28 @@ extern "C" ql_status qlinear_forward_a8(qlinear_t h, const void* x, void* y, int
 {
     if (!h || !x || !y || M < 1) return QL_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 15) return QL_ERR_INVALID_ARG;
-    if (M > 8 || M > h->gemv_max_m) return QL_ERR_UNSUPPORTED;          // the decode stage only
     if (device_timed_out(h)) return QL_ERR_DEVICE_TIMEOUT;
     const Layout& L = h->L;
+    if (M > h->gemv_max_m) {
+        // Prefill stage (Section 3.7): the quantisation kernel, then the integer matmul with output dequantisation.
+        // Built for the per-channel schemes on the CTA-pair kernel; the quantised activations live in the device's
+        // shared scratch (calls must be ordered against other users of it).
+        if (L.grouped || (L.K % 128) || !gemm_pair_applicable(L, M)) return QL_ERR_UNSUPPORTED;
+        const size_t xq_bytes = (((size_t)M * L.K + 255) / 256) * 256, arr = (((size_t)M * 4 + 255) / 256) * 256;
+        if (xq_bytes + 2 * arr > gemm_pair_scratch_bytes(h->num_sms)) return QL_ERR_UNSUPPORTED;
+        DeviceGuard guard(h->device);
+        if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        unsigned char* base = reinterpret_cast<unsigned char*>(h->dev->gemm_scratch);
+        signed char* xq = reinterpret_cast<signed char*>(base);
+        float* sx = reinterpret_cast<float*>(base + xq_bytes);
+        int32_t* rs = reinterpret_cast<int32_t*>(base + xq_bytes + arr);
+        quantize_activations_kernel<<<M, 256, 0, st>>>(static_cast<const __half*>(x), xq, sx, rs, M, L.K);
+        if (cudaGetLastError() != cudaSuccess) return QL_ERR_CUDA;
+        GemmPairLayers set{};
+        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y;
+        return gemm_pair_forward_i8(set, xq, sx, rs, M, st, h->device, h->pdl, h->num_sms);
+    }
     const GemvPlan pl = plan_gemv(L, h->n_rb, M, h->num_sms, false, true);
     if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
     DeviceGuard guard(h->device);
@@ -634,7 +653,7 @@ extern "C" ql_status qlinear_quantize_activations(const void* x, int8_t* xq, flo
     DeviceGuard guard(device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     quantize_activations_kernel<<<M, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __half*>(x),
-                                                                                reinterpret_cast<signed char*>(xq), scale, M, K);
+                                                                                reinterpret_cast<signed char*>(xq), scale, nullptr, M, K);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 

@@ -156,6 +156,17 @@ __device__ __forceinline__ void umma_f16_pair_lo(uint32_t tmem_d, uint32_t a_lo,
                  "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
                  ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128) : "memory");
 }
+// The integer form (kind::i8): A unsigned 8-bit, B signed 8-bit (which is which is in the instruction descriptor),
+// s32 accumulator in tensor memory, 32 k per instruction.
+__device__ __forceinline__ void umma_i8_pair_lo(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "mov.b64 da, {%1, %5};\n\t"
+                 "mov.b64 db, {%2, %5};\n\t"
+                 "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %3, p;\n\t}"
+                 ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHiSw128) : "memory");
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

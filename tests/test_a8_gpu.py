@@ -95,6 +95,57 @@ def test_a8_integer_path_is_bit_exact_when_no_rounding_is_left(P, torch, bits, g
     assert (y.view(np.uint16) == y16.view(np.uint16)).all()
 
 
+PREFILL = [
+    # (M, N, K, bits): per-channel schemes on the integer tensor-core path (K a multiple of 128, 256-channel tiles)
+    (129, 256, 128, 8), (300, 512, 1024, 8), (256, 256, 2304, 4), (700, 768, 1152, 4), (1024, 1024, 4096, 4), (2048, 256, 14336, 8),
+    (257, 1000, 512, 8),
+]
+
+
+@pytest.mark.parametrize("M,N,K,bits", PREFILL)
+def test_a8_prefill_parity(P, torch, M, N, K, bits):
+    """Prefill stage: quantisation kernel + kind::i8 matmul + output dequantisation against the same oracle."""
+    q, s, x = rand_case(7300 + N + K + M, M, N, K, bits, 0)
+    lin = P.QLinear.from_weights(q, s, bits, 0, device="cuda:0")
+    xd = torch.from_numpy(x).cuda()
+    y = lin.forward_a8(xd)
+    torch.cuda.synchronize()
+    assert lin.device_status() == (0, 0)
+    assert_a8(y.cpu().numpy(), x, q, s, 0)
+    assert torch.equal(y, lin.forward_a8(xd))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_a8_prefill_integer_path_is_bit_exact_when_no_rounding_is_left(P, torch, bits):
+    M, N, K = 300, 256, 512
+    rng = np.random.default_rng(4)
+    lo, hi = (-8, 7) if bits == 4 else (-128, 127)
+    q = rng.integers(lo, hi + 1, size=(N, K)).astype(np.int8)
+    q[:, 0], q[:, 1] = lo, hi
+    s = (2.0 ** rng.integers(-12, -8, size=(N, 1))).astype(np.float16)
+    ints = rng.integers(-127, 128, size=(M, K))
+    ints[:, 0], ints[:, 1] = 127, -127
+    x = (ints * (2.0 ** -rng.integers(0, 6, size=(M, 1)))).astype(np.float16)
+    lin = P.QLinear.from_weights(q, s, bits, 0, device="cuda:0")
+    y = lin.forward_a8(torch.from_numpy(x).cuda()).cpu().numpy()
+    _, _, xq, _, y16 = O.linear_int8_activations(x, q, s, 0)
+    assert (xq == ints).all()
+    assert (y.view(np.uint16) == y16.view(np.uint16)).all()
+
+
+@pytest.mark.parametrize("name,bits", [("q", 8), ("gate", 4), ("down", 4)])
+def test_a8_prefill_llama_shapes_full_size(P, torch, name, bits):
+    """The Llama3.1-8B shapes at M = 2048 in the paper's own schemes (q8 attention, per-channel int4 feed-forward)."""
+    layer = [l for l in C.LLAMA31_8B if l.name == name][0]
+    spec = C.LayerSpec(name, layer.N, layer.K, bits, 0, *((-8, 7) if bits == 4 else (-128, 127)))
+    q, s = C.layer_weights(7400, spec)
+    x = C.layer_activations(7400, spec, 2048)
+    lin = P.QLinear.from_weights(q, s, bits, 0, device="cuda:0")
+    y = lin.forward_a8(torch.from_numpy(x).cuda()).cpu().numpy()
+    for r0 in range(0, layer.N, 2048):                  # bounds the oracle's working set
+        assert_a8(y[:, r0:r0 + 2048], x, q[r0:r0 + 2048], s[r0:r0 + 2048], 0)
+
+
 def test_a8_zero_input_and_guard_bands(P, torch):
     q, s, x = rand_case(7100, 3, 200, 352, 4, 32)
     lin = P.QLinear.from_weights(q, s, 4, 32, device="cuda:0")
@@ -105,8 +156,8 @@ def test_a8_zero_input_and_guard_bands(P, torch):
     torch.cuda.synchronize()
     assert (buf[:guard] == -7.0).all() and (buf[-guard:] == -7.0).all()
     assert (y == 0).all()
-    with pytest.raises(P.QLinearError) as err:        # the decode stage only
-        lin.forward_a8(torch.zeros((9, 352), dtype=torch.float16, device="cuda"))
+    with pytest.raises(P.QLinearError) as err:        # prefill stage: per-channel schemes only
+        lin.forward_a8(torch.zeros((300, 352), dtype=torch.float16, device="cuda"))
     assert err.value.status == P.QL_ERR_UNSUPPORTED
 
 
