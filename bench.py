@@ -625,6 +625,7 @@ def main():
             if not args.no_configs:
                 line["configs"] += prefill_configs(torch, device, peaks, sidx, line)
                 line["fused_gating"] = gated_record(torch, device, peaks, sidx, ls)
+                line["int8_activations"] = a8_record(torch, device, peaks, sidx)
         # ---- CPU oracle beside it (bounded sample)
         if not args.no_cpu_baseline:
             rows = calibrate_rows(workload, M, 8.0)
@@ -708,6 +709,70 @@ def gated_record(torch, device, peaks, sidx, ls_main):
             rec["grouped_tflops"] = fl / 1e6 / rec["grouped_us"]
             rec["y_bytes_written"] = {"gated": 2 * M * layer.N, "grouped": 4 * M * layer.N}
         out[stage] = rec
+    return out
+
+
+def a8_record(torch, device, peaks, sidx):
+    """Int8 activations (paper Section 3.7) next to the fp16-activation kernels on the same weights: decode on the LM
+    head (quantisation fused into the kernel), prefill at M = 2048 on the Llama shapes in the paper's per-channel 8/4/4
+    scheme (quantisation kernel + integer tensor-core matmul; the times include the quantisation kernel)."""
+    import paper_2505_00232_b200 as P
+    out = {}
+    # ---- decode, LM head
+    w = C.CONFIG_5B
+    layer = w.layers[0]
+    desc = P.Desc(layer.N, layer.K, layer.bits, layer.group)
+    blob = torch.from_numpy(P.qlinear_pack(desc, *C.layer_weights(w.seed, layer, 0))).to(device)
+    lins = [P.QLinear(desc, blob), P.QLinear(desc, blob.clone())]
+    x = torch.from_numpy(C.layer_activations(w.seed, layer, 1, 0)).to(device)
+    y = torch.empty((1, layer.N), dtype=torch.float16, device=device)
+    rec = {"layer": f"lm_head {layer.N}x{layer.K} int4 group 32", "M": 1}
+    for name in ("f16", "a8"):
+        fn = (lambda cp: lins[cp].forward_raw(x.data_ptr(), y.data_ptr(), 1)) if name == "f16" else \
+             (lambda cp: lins[cp].forward_a8_raw(x.data_ptr(), y.data_ptr(), 1))
+        graph = capture_graph(torch, lambda i: fn(i % 2), 2)
+        for _ in range(3):
+            graph.replay()
+        ms, repeats, clocks = timed_region(torch, graph.replay, 2, sidx, 0.25)
+        us = ms * 1e3 / (2 * repeats)
+        rec[name] = {"us": us, "gbs": layer.weight_bytes / 1e3 / us, "frac_of_measured_peak": layer.weight_bytes / 1e3 / us / peaks["hbm_gbs"],
+                     "sm_mhz": clocks["sm_mhz"]}
+    out["decode"] = rec
+    del lins, blob
+    torch.cuda.empty_cache()
+    # ---- prefill, Llama shapes, per-channel 8/4/4
+    wl = C.by_name("llama31_8b_decode_pc4")
+    M = 2048
+    rows = []
+    tot = {"f16": 0.0, "a8": 0.0}
+    flops = 0
+    for li, layer in enumerate(wl.layers):
+        if layer.name in ("k", "v", "up"):
+            continue                                                      # same shapes as q / gate; k and v alone have too few tiles for this kernel
+        desc = P.Desc(layer.N, layer.K, layer.bits, layer.group)
+        blob = torch.from_numpy(P.qlinear_pack(desc, *C.layer_weights(wl.seed, layer, li))).to(device)
+        lins = [P.QLinear(desc, blob), P.QLinear(desc, blob.clone())]
+        x = torch.from_numpy(C.layer_activations(wl.seed, layer, M, li)).to(device)
+        y = torch.empty((M, layer.N), dtype=torch.float16, device=device)
+        r = {"layer": f"{layer.name} {layer.N}x{layer.K} int{layer.bits} per channel"}
+        for name in ("f16", "a8"):
+            fn = (lambda cp: lins[cp].forward_raw(x.data_ptr(), y.data_ptr(), M)) if name == "f16" else \
+                 (lambda cp: lins[cp].forward_a8_raw(x.data_ptr(), y.data_ptr(), M))
+
+            def block():
+                fn(0)
+                fn(1)
+            block()
+            ms, repeats, clocks = timed_region(torch, block, 2, sidx, 0.25)
+            us = ms * 1e3 / (2 * repeats)
+            r[name] = {"us": us, "tera_ops": layer.flops(M) / 1e6 / us, "sm_mhz": clocks["sm_mhz"]}
+            tot[name] += us
+        flops += layer.flops(M)
+        rows.append(r)
+        del lins, blob
+        torch.cuda.empty_cache()
+    out["prefill"] = {"M": M, "layers": rows, "sum": {k: {"us": v, "tera_ops": flops / 1e6 / v} for k, v in tot.items()},
+                      "note": "a8 = quantisation kernel + kind::i8 matmul; tera_ops counts 2*M*N*K for both"}
     return out
 
 

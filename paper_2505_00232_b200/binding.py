@@ -292,6 +292,9 @@ class QLinear:
                "qlinear_forward_a8")
         return out
 
+    def forward_a8_raw(self, x_ptr: int, y_ptr: int, M: int, stream=None) -> None:
+        _check(lib.qlinear_forward_a8(self._h, ctypes.c_void_p(x_ptr), ctypes.c_void_p(y_ptr), M, _stream_ptr(stream)), "qlinear_forward_a8")
+
     def forward_raw(self, x_ptr: int, y_ptr: int, M: int, stream=None) -> None:
         _check(lib.qlinear_forward(self._h, ctypes.c_void_p(x_ptr), ctypes.c_void_p(y_ptr), M, _stream_ptr(stream)),
                "qlinear_forward")
