@@ -126,12 +126,13 @@ def physical_gpu_index(local: int) -> int:
 class LayerSet:
     """`copies` independent weight copies of every layer of a workload, resident on one GPU."""
 
-    def __init__(self, workload, M, copies, device, distinct_copies=True, blobs=None):
+    def __init__(self, workload, M, copies, device, distinct_copies=True, blobs=None, act="fp16"):
         """blobs: optional {layer index: packed device tensor} to bind copy 0 to weights that are already
         resident (the paper's point: one resident copy serves both stages)."""
         import torch
         import paper_2505_00232_b200 as P
         self.P, self.torch, self.workload, self.M, self.copies = P, torch, workload, M, copies
+        self.act = act                        # "fp16": qlinear_forward; "int8": qlinear_forward_a8 (one call per layer)
         self.layers = workload.layers
         self.lin = [[None] * len(self.layers) for _ in range(copies)]
         self.blob0 = {}
@@ -174,7 +175,8 @@ class LayerSet:
     def step(self, cp, only=None):
         for li in range(len(self.layers)):
             if only is None or li in only:
-                self.lin[cp][li].forward_raw(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
+                fwd = self.lin[cp][li].forward_a8_raw if self.act == "int8" else self.lin[cp][li].forward_raw
+                fwd(self.x[li].data_ptr(), self.y[li].data_ptr(), self.M)
 
     _STAGE = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}
 
@@ -502,6 +504,8 @@ def main():
                     help="decode graph: one launch per layer (default: layers that read the same input, q/k/v and "
                          "gate/up, go out as one grouped call each, the data flow of a transformer layer)")
     ap.add_argument("--no-prefill", action="store_true", help="skip the prefill sub-measurement")
+    ap.add_argument("--act", default="fp16", choices=["fp16", "int8"],
+                    help="int8: the int8-activation entry point (paper Section 3.7), one call per layer")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-workload record (configs 1-5, LM head, q8, 8/4/4)")
     ap.add_argument("--prefill-steps", type=int, default=20)
@@ -535,7 +539,9 @@ def main():
         copies = args.copies or max(4, -(-3 * l2 // layer_bytes))
     else:
         copies = args.copies or max(1, -(-3 * l2 // (2 * layer_bytes)))
-    ls = LayerSet(workload, M, copies, device, distinct_copies=True)
+    ls = LayerSet(workload, M, copies, device, distinct_copies=True, act=args.act)
+    if args.act == "int8":
+        args.no_groups = True
     use_graph = (stage == "decode") and not args.no_graph
 
     # ---- main timed region: K steps (repeated back to back, see timed_region), barrier + synchronize on both

@@ -269,7 +269,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         for (int j = 0; tile_of(j, t, gl) && ok; ++j) {
             const int n_steps = pair_unit(t, p).nsteps;
             for (int it = 0; it < n_steps; ++it, ++gstep) {
-                if (!mbar_wait<true>(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
+                if (!mbar_wait(full_bar(s), par, abort_flag, 0x400 + s)) { ok = false; break; }
                 if (gstep >= NA) {
                     if (!mbar_wait(empty_bar(s_old), par_old, abort_flag, 0xB00 + s_old)) { ok = false; break; }
                     if (++s_old == NS) { s_old = 0; par_old ^= 1; }
@@ -348,14 +348,23 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
 #pragma unroll 1
                 for (int cc = 0; cc < ml; cc += 16) {
                     uint32_t r[16];
+                    // the 16 tokens' scales and row sums first (whole 64-byte lines; the arrays are padded to whole tiles)
+                    float sx[16];
+                    int rs[16];
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const float4 f = __ldg(reinterpret_cast<const float4*>(p.a8_scale + m0 + cc) + v);
+                        const int4 i = __ldg(reinterpret_cast<const int4*>(p.a8_rowsum + m0 + cc) + v);
+                        sx[4 * v] = f.x; sx[4 * v + 1] = f.y; sx[4 * v + 2] = f.z; sx[4 * v + 3] = f.w;
+                        rs[4 * v] = i.x; rs[4 * v + 1] = i.y; rs[4 * v + 2] = i.z; rs[4 * v + 3] = i.w;
+                    }
                     tmem_ld16(ta + (uint32_t)cc, r);
                     if (n < N) {
 #pragma unroll
                         for (int q = 0; q < 16; ++q)
                             if (cc + q < ml) {
-                                const int tok = m0 + cc + q;
-                                const float v = (float)((int)r[q] - OFF * p.a8_rowsum[tok]);
-                                yr[(int64_t)(cc + q) * N] = __float2half_rn(p.a8_scale[tok] * (sn * v));
+                                const float v = (float)((int)r[q] - OFF * rs[q]);
+                                yr[(int64_t)(cc + q) * N] = __float2half_rn(sx[q] * (sn * v));
                             }
                     }
                 }

@@ -605,7 +605,8 @@ extern "C" ql_status qlinear_forward_a8(qlinear_t h, const void* x, void* y, int
         // Built for the per-channel schemes on the CTA-pair kernel; the quantised activations live in the device's
         // shared scratch (calls must be ordered against other users of it).
         if (L.grouped || (L.K % 128) || !gemm_pair_applicable(L, M)) return QL_ERR_UNSUPPORTED;
-        const size_t xq_bytes = (((size_t)M * L.K + 255) / 256) * 256, arr = (((size_t)M * 4 + 255) / 256) * 256;
+        const size_t xq_bytes = (((size_t)M * L.K + 255) / 256) * 256;
+        const size_t arr = (size_t)((M + 255) / 256) * 256 * 4;             // per-token arrays padded to whole 256-token tiles
         if (xq_bytes + 2 * arr > gemm_pair_scratch_bytes(h->num_sms)) return QL_ERR_UNSUPPORTED;
         DeviceGuard guard(h->device);
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }

@@ -89,6 +89,7 @@ LLAMA31_8B_PC4 = tuple(l if l.bits == 8 else LayerSpec(l.name, l.N, l.K, 4, 0, -
 SCHEMES = (
     Workload("llama31_8b_decode_q8", 6, LLAMA31_8B_Q8, (1,), "decode"),
     Workload("llama31_8b_decode_pc4", 7, LLAMA31_8B_PC4, (1,), "decode"),
+    Workload("llama31_8b_prefill_pc4", 7, LLAMA31_8B_PC4, (2048,), "prefill"),
 )
 
 
