@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqlinear.so")
 SOURCES = ["qlinear.cu", "pack.cpp"]
-DEPS = SOURCES + ["layout.h", "dequant.cuh", "sm100_ptx.cuh", "embed.cuh", "gemv.cuh", "gemv_a8.cuh", "kv.cuh", "gemv_stream.cuh", "gemm.cuh", "gemm_pair.cuh", os.path.join("..", "..", "include", "qlinear.h")]
+DEPS = SOURCES + ["layout.h", "dequant.cuh", "sm100_ptx.cuh", "embed.cuh", "gemv.cuh", "gemv_a8.cuh", "kv.cuh", "gemv_stream.cuh", "gemm.cuh", "gemm_pair.cuh", "gemm_pair_ta.cuh", os.path.join("..", "..", "include", "qlinear.h")]
 
 
 def _stale() -> bool:
@@ -26,6 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-Xcompiler", "-fPIC,-O3,-fopenmp", "-shared", "-cudart", "static",
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lgomp"]
+    cmd[1:1] = os.environ.get("QL_EXTRA_NVCC_FLAGS", "").split()   # e.g. -DQL_TA_EXPERIMENT for timing experiments
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -352,6 +352,7 @@ struct GemmConfig {
     int force_split = 0;     // QLINEAR_GEMM_SPLIT: K parts of single-round layers in the CTA-pair kernel (0 = choose)
     int force_tb = 0;        // QLINEAR_GEMM_TB: token blocks per tile of the CTA-pair kernel (0 = choose)
     bool pair = true;        // QLINEAR_GEMM_PAIR=0 switches the CTA-pair kernel off
+    bool ta = true;          // QLINEAR_GEMM_TA=0 switches off the CTA-pair kernel that keeps the dequantised weights in tensor memory
 };
 GemmConfig& gemm_config();
 

@@ -193,7 +193,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        // The whole warp runs the loop (warp-uniform control flow: counters and descriptors stay in uniform
+        // registers); one elected lane issues.
+        if (rank == 0) {
             // f16 x f16 -> f32, or (integer form) u8 weights x s8 activations -> s32; both operands K-major, M = 256 per pair
             constexpr uint32_t idesc = (I8 ? (2u << 4) | (1u << 10) : (1u << 4)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
             const uint32_t a_lo0 = umma_desc_lo(a_addr(0)), b_lo0 = umma_desc_lo(xs_addr(0));
@@ -210,28 +212,31 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap x_map, const GemmParams p)
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(buf * BN);
                 for (int it = 0; it < n_steps; ++it) {
-                    // own A tile written (implies own x half landed) and the peer's likewise
                     // 16 local dequantise warps + the peer's relay lane: both A tiles written, both x halves landed
                     if (!mbar_wait_hot(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_lo = a_lo0 + (uint32_t)a * (kGemmATileBytes >> 4);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kStageBytes >> 4);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int tb = 0; tb < TB; ++tb) {
-                        const uint32_t d = tmem_d + (uint32_t)(tb * BN), bl = b_lo + (uint32_t)tb * (S::kXBlockBytes >> 4);
-                        if (I8) umma_i8_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
-                        else umma_f16_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
+                        for (int tb = 0; tb < TB; ++tb) {
+                            const uint32_t d = tmem_d + (uint32_t)(tb * BN), bl = b_lo + (uint32_t)tb * (S::kXBlockBytes >> 4);
+                            if (I8) umma_i8_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
+                            else umma_f16_pair_lo(d, a_lo, bl, idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k4 = 1; k4 < 4; ++k4) {                 // +32 bytes along K inside the swizzle row
-                            if (I8) umma_i8_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
-                            else umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                            for (int k4 = 1; k4 < 4; ++k4) {             // +32 bytes along K inside the swizzle row
+                                if (I8) umma_i8_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                                else umma_f16_pair_lo(d, a_lo + 2 * k4, bl + 2 * k4, idesc, 1u);
+                            }
                         }
+                        umma_commit_pair(empty_bar(s));                  // frees the TMA stage and the A slot in both CTAs
                     }
-                    umma_commit_pair(empty_bar(s));                      // frees the TMA stage and the A slot in both CTAs
+                    __syncwarp();
                     if (++s == NS) s = 0;
                     if (++a == NA) { a = 0; apar ^= 1; }
                 }
-                if (ok) umma_commit_pair(tfull_bar(buf));
+                if (ok && elect_one()) umma_commit_pair(tfull_bar(buf));
+                __syncwarp();
             }
         }
     } else if (warp < kPairFirstEpilogueWarp) {
@@ -487,6 +492,7 @@ struct GemmPairLayers {
     const Layout* L[kGemmMaxGroup];
     const uint8_t* blob[kGemmMaxGroup];
     void* y[kGemmMaxGroup];
+    const CUtensorMap* wmap[kGemmMaxGroup];      // packed body as 64-byte rows (tensor-memory form), or nullptr
     int n_rsb() const { int t = 0; for (int i = 0; i < n; ++i) t += L[i]->n_rsb; return t; }
 };
 

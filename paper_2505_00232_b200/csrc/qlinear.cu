@@ -30,6 +30,7 @@ __device__ unsigned int* g_status_host;
 #include "kv.cuh"
 #include "gemm.cuh"
 #include "gemm_pair.cuh"
+#include "gemm_pair_ta.cuh"
 
 using namespace ql;
 
@@ -73,6 +74,7 @@ void load_config()
     c.gemm.force_split = env_int("QLINEAR_GEMM_SPLIT", 0);
     c.gemm.force_tb = env_int("QLINEAR_GEMM_TB", 0);
     c.gemm.pair = env_int("QLINEAR_GEMM_PAIR", 1) != 0;
+    c.gemm.ta = env_int("QLINEAR_GEMM_TA", 1) != 0;
     c.generation = g_cfg.generation + 1;
     g_cfg = c;
     g_getenv_reads.fetch_add(1);
@@ -127,6 +129,8 @@ struct qlinear_s {
     GemvPlan gemv[9];          // cluster decode kernel, index = M (1..8)
     bool use_stream;
     int stream_P, stream_stages;
+    CUtensorMap wmap;          // the packed body as rows of 64 bytes (prefill kernel with the weights in tensor memory)
+    bool wmap_ok;
     DeviceState* dev;
 };
 
@@ -458,6 +462,7 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
     h->gemv_max_m = cfg.gemv_max_m;
     h->pdl = cfg.pdl;
     h->n_rb = (L.N + kRbRows - 1) / kRbRows;
+    h->wmap_ok = w_tensor_map(L, h->blob, &h->wmap);
     for (int M = 1; M <= 8; ++M) {
         h->gemv[M] = plan_gemv(L, h->n_rb, M, sms);
         if (h->gemv[M].grid <= 0 && M <= h->gemv_max_m) { delete h; return QL_ERR_UNSUPPORTED; }   // no decode plan fits this shape
@@ -502,8 +507,8 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (M <= h->gemv_max_m) return h->use_stream ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
     if (gemm_pair_applicable(h->L, M)) {
         GemmPairLayers set{};
-        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y;
-        return gemm_pair_forward(set, x, M, st, h->device, h->pdl, h->num_sms, h->dev->gemm_scratch, h->dev->gemm_counters);
+        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y; set.wmap[0] = h->wmap_ok ? &h->wmap : nullptr;
+        return gemm_pair_forward_auto(set, x, M, st, h->device, h->pdl, h->num_sms, h->dev->gemm_scratch, h->dev->gemm_counters);
     }
     return gemm_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
@@ -533,8 +538,11 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
             if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
             GemmPairLayers set{};
             set.n = n;
-            for (int i = 0; i < n; ++i) { set.L[i] = &hs[i]->L; set.blob[i] = hs[i]->blob; set.y[i] = ys[i]; }
-            return gemm_pair_forward(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
+            for (int i = 0; i < n; ++i) {
+                set.L[i] = &hs[i]->L; set.blob[i] = hs[i]->blob; set.y[i] = ys[i];
+                set.wmap[i] = hs[i]->wmap_ok ? &hs[i]->wmap : nullptr;
+            }
+            return gemm_pair_forward_auto(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
                                      hs[0]->dev->gemm_scratch, hs[0]->dev->gemm_counters);
         }
     }

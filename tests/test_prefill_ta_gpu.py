@@ -1,0 +1,108 @@
+"""Prefill kernel that keeps the dequantised weights in tensor memory (launches with at least one 256 x 256 tile per
+CTA pair): against the CPU oracle on ragged shapes of every scheme, and bit for bit against the shared-memory form of
+the same product, which a child process computes with the kernel switched off (the switch is read once per process).
+Both forms feed the tensor cores the same fp16 weights in the same k order, so their outputs must be identical."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+from oracle import qlinear_oracle as O
+from workloads import configs as C
+
+pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def P(_built_library):
+    import paper_2505_00232_b200 as P
+    return P
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    return torch
+
+
+# (M, N, K, bits, group): >= 74 tiles of 256 channels x 256 tokens each; ragged M, N and K tails; an odd number of
+# int8 chunks; a single k-step pair; grouped and per-channel int4; group sizes the packer expands to 32
+CASES = [
+    (1000, 4856, 1056, 4, 32), (777, 6400, 352, 8, 0), (2048, 2560, 2304, 4, 0), (520, 9728, 640, 4, 128),
+    (4096, 1280, 1024, 8, 0), (300, 19456, 128, 4, 64), (2047, 2816, 4096, 4, 32),
+]
+
+
+def case(seed, M, N, K, bits, group):
+    layer = C.LayerSpec("t", N, K, bits, group, *((-8, 7) if bits == 4 else (-128, 127)))
+    q, s = C.layer_weights(seed, layer)
+    return q, s, C.layer_activations(seed, layer, M)
+
+
+def run(P, torch, M, N, K, bits, group, seed):
+    q, s, x = case(seed, M, N, K, bits, group)
+    desc = P.Desc(N, K, bits, group)
+    lin = P.QLinear(desc, torch.from_numpy(P.qlinear_pack(desc, q, s)).cuda())
+    y = lin.forward(torch.from_numpy(x).cuda())
+    torch.cuda.synchronize()
+    st, detail = lin.device_status()
+    assert st == 0, f"device status {st} detail {detail:#x}"
+    return q, s, x, y.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,N,K,bits,group", CASES)
+def test_parity_against_oracle(P, torch, M, N, K, bits, group):
+    q, s, x, y = run(P, torch, M, N, K, bits, group, 7000 + M + N)
+    assert np.isfinite(y.astype(np.float32)).all()
+    rows = 2048
+    d2 = y2 = worst = 0.0
+    for r0 in range(0, N, rows):
+        y64, A, _ = O.linear(x, q[r0:r0 + rows], s[r0:r0 + rows], group)
+        d = y[:, r0:r0 + rows].astype(np.float64) - y64
+        d2 += float((d * d).sum())
+        y2 += float((y64 * y64).sum())
+        with np.errstate(divide="ignore", invalid="ignore"):
+            worst = max(worst, float(np.where(A > 0, np.abs(d) / A, np.where(d == 0, 0.0, np.inf)).max()))
+    assert (d2 / y2) ** 0.5 <= O.REL_L2_TOL and worst <= O.ELEM_TOL, f"rel_l2={(d2 / y2) ** 0.5:.3e} worst={worst:.3e}"
+
+
+CHILD = """
+import sys, numpy as np, torch
+sys.path.insert(0, {root!r})
+import paper_2505_00232_b200 as P
+from tests.test_prefill_ta_gpu import CASES, run
+np.savez({out!r}, **{{str(i): run(P, torch, *c, 7000 + c[0] + c[1])[3] for i, c in enumerate(CASES)}})
+"""
+
+
+def test_bit_identical_to_the_shared_memory_form(P, torch, tmp_path):
+    out = str(tmp_path / "shared_memory_form.npz")
+    env = dict(os.environ, QLINEAR_GEMM_TA="0")
+    subprocess.run([sys.executable, "-c", CHILD.format(root=ROOT, out=out)], check=True, env=env, cwd=ROOT, timeout=600)
+    ref = np.load(out)
+    for i, c in enumerate(CASES):
+        y = run(P, torch, *c, 7000 + c[0] + c[1])[3]
+        assert np.array_equal(y.view(np.uint16), ref[str(i)].view(np.uint16)), f"case {c}"
+
+
+def test_guard_band_around_y(P, torch):
+    """The output tile leaves through bulk copies of whole 256-byte rows: nothing outside [M, N] may be written."""
+    M, N, K, bits, group = 300, 19448, 128, 4, 32                        # ragged last row super-block (120 channels)
+    q, s, x = case(11, M, N, K, bits, group)
+    desc = P.Desc(N, K, bits, group)
+    lin = P.QLinear(desc, torch.from_numpy(P.qlinear_pack(desc, q, s)).cuda())
+    pad = 4096
+    buf = torch.full((pad + M * N + pad,), -7.0, dtype=torch.float16, device="cuda")
+    xd = torch.from_numpy(x).cuda()
+    lin.forward_raw(xd.data_ptr(), buf.data_ptr() + 2 * pad, M)
+    torch.cuda.synchronize()
+    h = buf.cpu().numpy()
+    assert (h[:pad] == -7.0).all() and (h[pad + M * N:] == -7.0).all()
+    y = h[pad:pad + M * N].reshape(M, N)
+    y64, A, _ = O.linear(x, q, s, group)
+    ok, rel, worst = O.check_against(y, y64, A)
+    assert ok, f"rel_l2={rel:.3e} worst={worst:.3e}"
