@@ -43,7 +43,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # capture each, summarised with its command under profiles/), averaged over the launches this file times.
 NCU_TRAFFIC_BYTES = {
     ("llama31_8b_decode", 1): (66.095104e6 + 0.455936e6 + 33.085440e6) / 2,     # gate+up and down launches
-    ("llama31_8b_prefill", 2048): (73.6e6 + 73.6e6 + 95.9e6) / 3,            # gate, up, down (reads + y write-back)
+    # gemm_pair_ta_kernel: gate + up grouped (83.06 + 82.21 MB, halved per layer) and down (146.67 + 12.78 MB)
+    ("llama31_8b_prefill", 2048): (82.64e6 + 82.64e6 + 159.44e6) / 3,
 }
 
 
@@ -453,7 +454,7 @@ def decode_roofline(torch, ls, workload, M, peaks, use_graph, grouped, sampler_i
             "launches": per_launch, "frac_of_nominal_8tbs": achieved / 8000.0}
 
 
-def prefill_roofline(torch, ls, workload, M, peaks, sampler_index, kernel_name="gemm_pair_kernel<int4, grouped>"):
+def prefill_roofline(torch, ls, workload, M, peaks, sampler_index, kernel_name="gemm_pair_ta_kernel<int4, grouped>"):
     ids4 = [i for i, l in enumerate(workload.layers) if l.bits == 4] or list(range(len(workload.layers)))
     ms, _ = kernel_time(torch, ls, ids4, False, False, sampler_index)
     flops = sum(workload.layers[i].flops(M) for i in ids4) / len(ids4)

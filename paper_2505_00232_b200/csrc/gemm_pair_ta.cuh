@@ -208,6 +208,9 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     cluster_sync_all();                                                  // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // The next kernel in the stream may move onto SMs this grid has left (the last, partial round of tiles) and set up
+    // there; whatever it reads of this grid's output comes after its own griddepcontrol.wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // Relay (peer CTA): "A slot written, x tile landed" -> one arrive on the leader's afull barrier; two threads (warps 1 and
     // 3 of the peer) take alternate steps.  The arrive is RELAXED: with release semantics at cluster scope it took about a
