@@ -147,7 +147,12 @@ struct DequantRowTa {
 };
 
 // Warp roles: 0 weight producer, 1 MMA issuer (leader) / relay (peer), 2 x producer, 3 spare, 4..27 dequantise (4..19 also epilogue).
-template <int BITS, bool GROUPED>
+// GATED: the launch serves two layers of equal shape, gate (0) and up (1).  A cluster runs the gate tile and then the up
+// tile of the same (row super-block pair, token block) position.  The gate tile's epilogue leaves fp16(act(gate)) in
+// the shared output tile (nothing is sent to memory); the up tile's epilogue multiplies what it finds there by the up
+// projection, every thread reading back the values it wrote itself, and only that product goes to y (paper Section
+// 3.6).  n_tiles then counts positions of ONE layer.
+template <int BITS, bool GROUPED, bool GATED = false>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
 {
@@ -180,7 +185,16 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     const uint32_t rank = cluster_ctarank();                             // 0 = leader
     const int n_mblk = (p.M + BN - 1) / BN;
     const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
+    // the j-th unit of work of this cluster: a tile and, in the gated form, which of the two layers
+    auto unit = [&](int j, int& tile, int& gl) {
+        tile = first_tile + (GATED ? j >> 1 : j) * tile_stride;
+        gl = GATED ? (j & 1) : 0;
+        return tile < p.n_tiles;
+    };
+    int n_units = 0;
+    for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) n_units += GATED ? 2 : 1;
     const int n_steps = p.n_ksteps;
+    const int total_steps = n_units * n_steps;
     const int w_rows = p.block_bytes >> 6;                               // 64-byte rows per packed block
 
     if (threadIdx.x == 0) {
@@ -219,9 +233,6 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     // complete_tx) before the peer's own barrier completed, and they are read by the peer's own tensor core, which the
     // leader's MMA instruction starts only after it has seen this arrive.  Only the signal travels.
     auto relay = [&](int r) {
-        int n_my = 0;
-        for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) ++n_my;
-        const int total_steps = n_my * n_steps;
         int a = r;
         uint32_t apar = 0;
         for (int g = r; g < total_steps; g += 2) {
@@ -239,9 +250,10 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             int s = 0, issued = 0;
             uint32_t par = 1;
             bool ok = true;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+            int tile, gl;
+            for (int j = 0; ok && unit(j, tile, gl); ++j) {
                 int rsb = 2 * (tile / n_mblk) + (int)rank;
-                const int ly = pair_layer(p, rsb);
+                const int ly = GATED ? gl : pair_layer(p, rsb);
                 const int row0 = rsb * p.n_kc * w_rows;
                 const CUtensorMap* wm = &maps.w[ly];
                 for (int it = 0; it < n_steps; ++it) {
@@ -266,7 +278,8 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             abort_flag[3] = 1;
             int s = 0, g = 0;
             bool ok = true;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride) {
+            int tile, gl;
+            for (int j = 0; ok && unit(j, tile, gl); ++j) {
                 const int m0 = (tile % n_mblk) * BN + 128 * (int)rank;   // this CTA's 128 tokens
                 for (int it = 0; it < n_steps; ++it, ++g) {
                     // stage s was last used by step g - NX, whose MMAs signal A-slot barrier (g - NX) % NA; by then the
@@ -296,8 +309,8 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             int s = 0, a = 0;
             uint32_t apar = 0;
             bool ok = true;
-            int j = 0;
-            for (int tile = first_tile; tile < p.n_tiles && ok; tile += tile_stride, ++j) {
+            int tile, gl;
+            for (int j = 0; ok && unit(j, tile, gl); ++j) {
                 if (!mbar_wait_hot(tempty_bar, (uint32_t)(j & 1) ^ 1, abort_flag, 0x800)) { ok = false; break; }
                 tc_fence_after();
                 for (int it = 0; it < n_steps; ++it) {
@@ -340,22 +353,27 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
         unsigned char* out_ptr = base_ptr + S::kOutOffset;
         const int grp_thread = quarter * 32 + lane;                      // 0..127 inside the group of four warps
         auto epilogue = [&](int j) {
-            const int tile = first_tile + j * tile_stride;
+            int tile, gl;
+            unit(j, tile, gl);
             int rsb = 2 * (tile / n_mblk) + (int)rank;
-            const int ly = pair_layer(p, rsb);
+            const int ly = GATED ? 0 : pair_layer(p, rsb);
             const int N = p.lN[ly];
             const int m0 = (tile % n_mblk) * BN + 64 * wi;
-            // the bulk copies of the previous tile have read their rows of the output tile
-            if (grp_thread < 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(grp_bar(wi, 0));
-            bool live = mbar_wait(grp_bar(wi, 0), (uint32_t)(j & 1), abort_flag, 0xC00 + wi);
+            const uint32_t gpar = (uint32_t)(GATED ? j >> 1 : j) & 1;   // phase of the group barriers: once per output tile
+            bool live = true;
+            if (!GATED || gl == 0) {
+                // the bulk copies of the previous output tile have read their rows of the shared tile
+                if (grp_thread < 64) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(grp_bar(wi, 0));
+                live = mbar_wait(grp_bar(wi, 0), gpar, abort_flag, 0xC00 + wi);
+            }
             live = live && mbar_wait(tfull_bar, (uint32_t)(j & 1), abort_flag, 0x500);
             if (live) {
                 tc_fence_after();
                 const int n = rsb * kRsbRows + quarter * 32 + lane;
                 float scale = 1.f;
-                if (!GROUPED && n < N) scale = __half2float(p.lscales[ly][n]);
+                if (!GROUPED && n < N) scale = __half2float(p.lscales[GATED ? gl : ly][n]);
                 const uint32_t taddr = tmem_base + lane_base + (uint32_t)(64 * wi);
                 __half* orow = reinterpret_cast<__half*>(out_ptr + (64 * wi) * 256) + grp_thread;
 #pragma unroll
@@ -369,14 +387,23 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                     }
                     if (!(QL_TA_EXP & 2)) {
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) orow[(cc + q) * 128] = __float2half_rn(__uint_as_float(r[q]) * scale);
+                        for (int q = 0; q < 32; ++q) {
+                            float v = __uint_as_float(r[q]) * scale;
+                            if (GATED && gl == 0) v = gate_activation(v, p.act);
+                            if (GATED && gl == 1) v *= __half2float(orow[(cc + q) * 128]);   // this thread's own act(gate)
+                            orow[(cc + q) * 128] = __float2half_rn(v);
+                        }
                     }
                 }
                 fence_async_smem();
             }
+            if (GATED && gl == 0) {                                      // the product is sent when the up tile is done
+                if (!live) ok = false;
+                return;
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(grp_bar(wi, 1));
-            live = mbar_wait(grp_bar(wi, 1), (uint32_t)(j & 1), abort_flag, 0xC10 + wi) && live;
+            live = mbar_wait(grp_bar(wi, 1), gpar, abort_flag, 0xC10 + wi) && live;
             if (live && grp_thread < 64 && m0 + grp_thread < p.M && !(QL_TA_EXP & 2)) {
                 const int n0 = rsb * kRsbRows;
                 const uint32_t bytes = (uint32_t)min(kRsbRows, N - n0) * 2;
@@ -395,9 +422,6 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
         };
 
         // The k-steps of all tiles of this cluster are numbered through (g); this warp takes g = my_turn, my_turn + 3, ...
-        int n_my = 0;
-        for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) ++n_my;
-        const int total_steps = n_my * n_steps;
         const int forced = min(S::kEarlySteps, n_steps - 1);
         int s = my_turn, a = my_turn;                                    // W stage and A slot of step g (my_turn < NW, NA)
         uint32_t wpar = 0, apar = 1;                                     // A slots start out free
@@ -429,7 +453,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             s += 3; if (s >= NW) { s -= NW; wpar ^= 1; }
             a += 3; if (a >= NA) { a -= NA; apar ^= 1; }
         }
-        while (epi_warp && ok && next_epi < n_my) { epilogue(next_epi); ++next_epi; }
+        while (epi_warp && ok && next_epi < n_units) { epilogue(next_epi); ++next_epi; }
         asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");        // y written before the kernel ends
     }
 
@@ -444,15 +468,16 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
 
 // The tensor-memory form takes whole tiles only (no K split, 256-token tiles, plain output): the launches with at
 // least one tile per cluster.
-template <int BITS, bool GROUPED>
-ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms)
+// act < 0: the plain form.  act >= 0: the gated form, set = {gate, up} of equal shape, y[0] the output.
+template <int BITS, bool GROUPED, bool GATED = false>
+ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms, int act = -1)
 {
     using S = GemmTaSmem<BITS>;
     const Layout& L = *set.L[0];
     TaMaps maps;
     if (!x_tensor_map(x, L.K, M, 128, &maps.x)) return QL_ERR_CUDA;
     for (int i = 0; i < kGemmMaxGroup; ++i) maps.w[i] = *set.wmap[i < set.n ? i : 0];
-    auto kern = gemm_pair_ta_kernel<BITS, GROUPED>;
+    auto kern = gemm_pair_ta_kernel<BITS, GROUPED, GATED>;
     static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
@@ -472,9 +497,11 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
         prm.rsb_end[i] = n_rsb;
     }
     prm.n_layers = set.n;
+    prm.act = act;
 #ifdef QL_TA_EXPERIMENT
-    prm.act = getenv("QLINEAR_EXP") ? atoi(getenv("QLINEAR_EXP")) : 0;
+    if (!GATED) prm.act = getenv("QLINEAR_EXP") ? atoi(getenv("QLINEAR_EXP")) : 0;
 #endif
+    if (GATED) n_rsb = L.n_rsb;                                          // work units count positions of one layer
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
@@ -505,12 +532,12 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
     return QL_OK;
 }
 
-inline bool gemm_pair_ta_applicable(const GemmPairLayers& set, int M, int num_sms)
+inline bool gemm_pair_ta_applicable(const GemmPairLayers& set, int M, int num_sms, bool gated = false)
 {
     if (!gemm_config().ta || M <= 128) return false;
     for (int i = 0; i < set.n; ++i)
         if (!set.wmap[i]) return false;
-    return (set.n_rsb() / 2) * ((M + 255) / 256) >= num_sms / 2;
+    return ((gated ? set.L[0]->n_rsb : set.n_rsb()) / 2) * ((M + 255) / 256) >= num_sms / 2;
 }
 
 inline ql_status gemm_pair_ta_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms)
@@ -519,6 +546,15 @@ inline ql_status gemm_pair_ta_forward(const GemmPairLayers& set, const void* x, 
     if (L.bits == 8) return gemm_pair_ta_launch<8, false>(set, x, M, st, device, pdl, num_sms);
     if (L.grouped) return gemm_pair_ta_launch<4, true>(set, x, M, st, device, pdl, num_sms);
     return gemm_pair_ta_launch<4, false>(set, x, M, st, device, pdl, num_sms);
+}
+
+// Gated form: set = {gate, up}, both pair-applicable and of equal shape; y[0] receives act(gate) * up.
+inline ql_status gemm_pair_ta_forward_gated(const GemmPairLayers& set, const void* x, int M, int act, cudaStream_t st, int device, bool pdl, int num_sms)
+{
+    const Layout& L = *set.L[0];
+    if (L.bits == 8) return gemm_pair_ta_launch<8, false, true>(set, x, M, st, device, pdl, num_sms, act);
+    if (L.grouped) return gemm_pair_ta_launch<4, true, true>(set, x, M, st, device, pdl, num_sms, act);
+    return gemm_pair_ta_launch<4, false, true>(set, x, M, st, device, pdl, num_sms, act);
 }
 
 // The CTA-pair prefill call: the tensor-memory form where it applies, else the shared-memory form.

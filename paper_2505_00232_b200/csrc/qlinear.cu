@@ -573,8 +573,9 @@ extern "C" ql_status qlinear_forward_gated(qlinear_t hg, qlinear_t hu, const voi
     } else if (M > hg->gemv_max_m && gemm_pair_applicable(a, M)) {       // prefill: both accumulators of the CTA-pair kernel
         GemmPairLayers set{};
         set.n = 2;
-        set.L[0] = &hg->L; set.blob[0] = hg->blob; set.y[0] = y;
-        set.L[1] = &hu->L; set.blob[1] = hu->blob; set.y[1] = y;
+        set.L[0] = &hg->L; set.blob[0] = hg->blob; set.y[0] = y; set.wmap[0] = hg->wmap_ok ? &hg->wmap : nullptr;
+        set.L[1] = &hu->L; set.blob[1] = hu->blob; set.y[1] = y; set.wmap[1] = hu->wmap_ok ? &hu->wmap : nullptr;
+        if (gemm_pair_ta_applicable(set, M, hg->num_sms, true)) return gemm_pair_ta_forward_gated(set, x, M, act, st, hg->device, hg->pdl, hg->num_sms);
         return gemm_pair_forward_gated(set, x, M, act, st, hg->device, hg->pdl, hg->num_sms);
     }
     // Unfused: the two projections into the device's shared scratch, then the element-wise product.
