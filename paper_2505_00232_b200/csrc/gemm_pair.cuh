@@ -483,7 +483,8 @@ inline int gemm_pair_split(int tiles /* of the last, partial round */, int n_kst
 // (at least 40 MB: the same buffer holds the int8 activations of the integer form, up to M x K = 2048 x 14336, and
 // the two projections of the unfused gating route)
 inline size_t gemm_pair_scratch_bytes(int num_sms) { return std::max<size_t>((size_t)(num_sms / 2) * 2 * 256 * 128 * sizeof(float), (size_t)40 << 20); }
-inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 8; }
+// (the tensor-memory form counts arrivals per (tile, CTA, 16 epilogue warps) for up to num_sms / 4 split tiles)
+inline size_t gemm_pair_counter_count(int num_sms) { return (size_t)(num_sms / 2) * 32; }
 
 // The layers of one launch: all read the same x and agree in K and scheme; each has an even number of row
 // super-blocks.  L is the layout of the first one (K, chunking and scheme are taken from it).

@@ -185,15 +185,21 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     const uint32_t rank = cluster_ctarank();                             // 0 = leader
     const int n_mblk = (p.M + BN - 1) / BN;
     const int first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;   // tile = (rsb pair, token block)
+    // K split (p.split = 2 or 4 parts per tile; launches with so few tiles that every cluster then has ONE unit of work):
+    // work unit v = tile * split + part, this cluster's part covers k-steps [it_base, it_base + n_steps) of its tile
+    const int P = GATED ? 1 : p.split;
+    const int part = P > 1 ? first_tile % P : 0;
+    const int it_base = part * p.n_ksteps / P;
+    const int n_steps = (part + 1) * p.n_ksteps / P - it_base;          // k-steps per unit of work of this cluster
     // the j-th unit of work of this cluster: a tile and, in the gated form, which of the two layers
     auto unit = [&](int j, int& tile, int& gl) {
-        tile = first_tile + (GATED ? j >> 1 : j) * tile_stride;
+        const int v = first_tile + (GATED ? j >> 1 : j) * tile_stride;
+        tile = P > 1 ? v / P : v;
         gl = GATED ? (j & 1) : 0;
-        return tile < p.n_tiles;
+        return v < p.n_tiles * P;
     };
     int n_units = 0;
-    for (int tile = first_tile; tile < p.n_tiles; tile += tile_stride) n_units += GATED ? 2 : 1;
-    const int n_steps = p.n_ksteps;
+    for (int v = first_tile; v < p.n_tiles * P; v += tile_stride) n_units += GATED ? 2 : 1;
     const int total_steps = n_units * n_steps;
     const int w_rows = p.block_bytes >> 6;                               // 64-byte rows per packed block
 
@@ -259,7 +265,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                 for (int it = 0; it < n_steps; ++it) {
                     if (!mbar_wait(wempty_bar(s), par, abort_flag, 0x100 + s)) { ok = false; break; }
                     mbar_expect_tx(wfull_bar(s), W_BOX_BYTES);
-                    tma_load_2d(wpk_addr(s), wm, 0, row0 + it * CHUNKS * w_rows, wfull_bar(s));
+                    tma_load_2d(wpk_addr(s), wm, 0, row0 + (it_base + it) * CHUNKS * w_rows, wfull_bar(s));
                     ++issued;
                     if (++s == NW) { s = 0; par ^= 1; }
                 }
@@ -289,7 +295,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                         if (!mbar_wait(aempty_bar(ao), (uint32_t)((g - NX) / NA) & 1, abort_flag, 0x180 + ao)) { ok = false; break; }
                     }
                     mbar_expect_tx(afull_bar(g % NA), S::kXBytes);
-                    tma_load_2d(xs_addr(s), &maps.x, it * kGemmKStep, m0, afull_bar(g % NA));
+                    tma_load_2d(xs_addr(s), &maps.x, (it_base + it) * kGemmKStep, m0, afull_bar(g % NA));
                     if (++s == NX) s = 0;
                 }
             }
@@ -352,9 +358,65 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
         const uint32_t out_addr = base + S::kOutOffset;
         unsigned char* out_ptr = base_ptr + S::kOutOffset;
         const int grp_thread = quarter * 32 + lane;                      // 0..127 inside the group of four warps
+        // K-split tile: every part parks its fp32 accumulator in the device's scratch ([token][channel], a warp writes
+        // 128 contiguous bytes per token), frees the accumulator and counts itself in; the part that arrives last adds all
+        // parts in part order (fixed order, no float atomics, nobody waits) and stores y.
+        auto split_epilogue = [&](int j, int tile) {
+            int rsb = 2 * (tile / n_mblk) + (int)rank;
+            const int ly = pair_layer(p, rsb);
+            const int N = p.lN[ly];
+            const int m0 = (tile % n_mblk) * BN + 64 * wi;
+            float* slab0 = p.scratch + ((int64_t)((tile * P) * 2 + (int)rank) * BN + 64 * wi) * 128 + grp_thread;   // part 0
+            const int64_t part_stride = (int64_t)2 * BN * 128;
+            unsigned int* cnt = p.counters + ((tile * 2 + (int)rank) * 4 + wi) * 4 + quarter;
+            if (!mbar_wait(tfull_bar, (uint32_t)(j & 1), abort_flag, 0x500)) { ok = false; return; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + lane_base + (uint32_t)(64 * wi);
+            float* mine = slab0 + part * part_stride;
+#pragma unroll 1
+            for (int cc = 0; cc < 64; cc += 16) {
+                uint32_t r[16];
+                tmem_ld16(taddr + (uint32_t)cc, r);
+#pragma unroll
+                for (int q = 0; q < 16; ++q) __stcg(mine + (cc + q) * 128, __uint_as_float(r[q]));
+            }
+            tc_fence_before();
+            __threadfence();
+            __syncwarp();
+            unsigned int old = 0;
+            if (lane == 0) { mbar_arrive_remote(tempty_bar, 0); old = atomicAdd(cnt, 1u); }
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if ((int)old != P - 1) return;
+            __threadfence();
+            const int n = rsb * kRsbRows + quarter * 32 + lane;
+            float scale = 1.f;
+            if (!GROUPED && n < N) scale = __half2float(p.lscales[ly][n]);
+            __half* yrow = p.ly[ly] + (int64_t)m0 * N + n;
+            const int m_left = min(64, p.M - m0);
+#pragma unroll 1
+            for (int cc = 0; cc < m_left; cc += 8) {
+                float acc[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) acc[q] = __ldcg(slab0 + (cc + q) * 128);
+                for (int pp = 1; pp < P; ++pp) {
+                    float v[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) v[q] = __ldcg(slab0 + pp * part_stride + (cc + q) * 128);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc[q] += v[q];
+                }
+                if (n < N) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (cc + q < m_left) yrow[(int64_t)(cc + q) * N] = __float2half_rn(acc[q] * scale);
+                }
+            }
+            if (lane == 0) *cnt = 0;                                     // ready for the next launch
+        };
         auto epilogue = [&](int j) {
             int tile, gl;
             unit(j, tile, gl);
+            if (P > 1) { split_epilogue(j, tile); return; }
             int rsb = 2 * (tile / n_mblk) + (int)rank;
             const int ly = GATED ? 0 : pair_layer(p, rsb);
             const int N = p.lN[ly];
@@ -466,11 +528,26 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     }
 }
 
-// The tensor-memory form takes whole tiles only (no K split, 256-token tiles, plain output): the launches with at
-// least one tile per cluster.
+// The tensor-memory form: 256-token tiles, whole tiles dealt out round-robin, or (fewer tiles than half the CTA pairs)
+// 2 or 4 K parts per tile that meet in the device's scratch.
+// K parts per tile for a launch of `tiles` tiles: 1 unless the tiles would leave half of the CTA pairs (or more) idle.
+inline int gemm_pair_ta_split(int tiles, int n_ksteps, int num_sms, bool have_scratch)
+{
+    const int clusters = num_sms / 2;
+    int split = 1;
+    if (!have_scratch || tiles >= clusters) return 1;
+    if (gemm_config().force_split > 0) split = gemm_config().force_split >= 4 ? 4 : gemm_config().force_split >= 2 ? 2 : 1;
+    else if (tiles * 4 <= clusters) split = 4;
+    else if (tiles * 2 <= clusters) split = 2;
+    while (split > 1 && (n_ksteps / split < 8 || tiles * split > clusters)) split >>= 1;
+    return split;
+}
+
 // act < 0: the plain form.  act >= 0: the gated form, set = {gate, up} of equal shape, y[0] the output.
+// scratch / counters: the device's shared fp32 scratch and arrival counters for the K-split case (null: no split).
 template <int BITS, bool GROUPED, bool GATED = false>
-ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms, int act = -1)
+ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms, int act = -1,
+                              float* scratch = nullptr, unsigned int* counters = nullptr)
 {
     using S = GemmTaSmem<BITS>;
     const Layout& L = *set.L[0];
@@ -507,9 +584,12 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
     prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
     prm.n_rsb = n_rsb;
     prm.n_tiles = (n_rsb / 2) * ((M + 255) / 256);
-    prm.split = 1;
+    prm.split = GATED ? 1 : gemm_pair_ta_split(prm.n_tiles, prm.n_ksteps, num_sms, scratch && counters);
+    prm.scratch = scratch;
+    prm.counters = counters;
     prm.n_whole = prm.n_tiles;
-    const int n_clusters = prm.n_tiles < num_sms / 2 ? prm.n_tiles : num_sms / 2;
+    const int units = prm.n_tiles * prm.split;
+    const int n_clusters = units < num_sms / 2 ? units : num_sms / 2;
 
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(2 * n_clusters);
@@ -537,15 +617,24 @@ inline bool gemm_pair_ta_applicable(const GemmPairLayers& set, int M, int num_sm
     if (!gemm_config().ta || M <= 128) return false;
     for (int i = 0; i < set.n; ++i)
         if (!set.wmap[i]) return false;
-    return ((gated ? set.L[0]->n_rsb : set.n_rsb()) / 2) * ((M + 255) / 256) >= num_sms / 2;
+    // the gated form needs a whole number of positions per round of the grid's clusters to be worth it; the plain form
+    // takes every launch (few tiles: fewer clusters, or a K split through the device scratch)
+    return !gated || (set.L[0]->n_rsb / 2) * ((M + 255) / 256) >= num_sms / 2;
 }
 
-inline ql_status gemm_pair_ta_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms)
+inline ql_status gemm_pair_ta_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms,
+                                      float* scratch, unsigned int* counters)
 {
     const Layout& L = *set.L[0];
-    if (L.bits == 8) return gemm_pair_ta_launch<8, false>(set, x, M, st, device, pdl, num_sms);
-    if (L.grouped) return gemm_pair_ta_launch<4, true>(set, x, M, st, device, pdl, num_sms);
-    return gemm_pair_ta_launch<4, false>(set, x, M, st, device, pdl, num_sms);
+    // a caller that keeps its outputs in the scratch itself (the unfused gating route) gets no K split
+    const unsigned char* s0 = reinterpret_cast<const unsigned char*>(scratch);
+    for (int i = 0; i < set.n && scratch; ++i) {
+        const unsigned char* y = static_cast<const unsigned char*>(set.y[i]);
+        if (y >= s0 && y < s0 + gemm_pair_scratch_bytes(num_sms)) scratch = nullptr;
+    }
+    if (L.bits == 8) return gemm_pair_ta_launch<8, false>(set, x, M, st, device, pdl, num_sms, -1, scratch, counters);
+    if (L.grouped) return gemm_pair_ta_launch<4, true>(set, x, M, st, device, pdl, num_sms, -1, scratch, counters);
+    return gemm_pair_ta_launch<4, false>(set, x, M, st, device, pdl, num_sms, -1, scratch, counters);
 }
 
 // Gated form: set = {gate, up}, both pair-applicable and of equal shape; y[0] receives act(gate) * up.
@@ -561,7 +650,7 @@ inline ql_status gemm_pair_ta_forward_gated(const GemmPairLayers& set, const voi
 inline ql_status gemm_pair_forward_auto(const GemmPairLayers& set, const void* x, int M, cudaStream_t st,
                                         int device, bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
-    if (gemm_pair_ta_applicable(set, M, num_sms)) return gemm_pair_ta_forward(set, x, M, st, device, pdl, num_sms);
+    if (gemm_pair_ta_applicable(set, M, num_sms)) return gemm_pair_ta_forward(set, x, M, st, device, pdl, num_sms, scratch, counters);
     return gemm_pair_forward(set, x, M, st, device, pdl, num_sms, scratch, counters);
 }
 
