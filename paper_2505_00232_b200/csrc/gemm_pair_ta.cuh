@@ -50,15 +50,18 @@ constexpr int kTaEpilogueWarps = 16;
 constexpr int kTaSlotCols = 32;              // 64 k of fp16
 constexpr int kTaAccCols = 256;
 
-template <int BITS>
+// I8: the integer form (int8 activations, kind::i8): a k-step is 128 k, i.e. again 128 bytes per x row and 32 columns per A slot.
+template <int BITS, bool I8 = false>
 struct GemmTaSmem {
     // Two rings, because the two operands are needed at different times: the packed weights of a k-step are needed
     // early (they still have to be dequantised), its x tile only when the MMA is issued.  A deep ring of small
     // weight stages lets the dequantise warps run ahead; the x ring only has to cover the TMA latency.
     static constexpr int kXBytes = 128 * 128;                            // this CTA's 128 tokens x 64 k
-    static constexpr int kXStages = 7;                                   // <= kASlots: the x producer reads "stage free" off the A-slot barrier
-    static constexpr int kWBytes = BITS == 4 ? 5120 : 8192;              // packed block(s) of one k-step
-    static constexpr int kWStages = BITS == 4 ? 9 : 6;
+    static constexpr int kKStep = I8 ? 128 : kGemmKStep;
+    static constexpr int kXStages = (I8 && BITS == 8) ? 6 : 7;           // <= kASlots: the x producer reads "stage free" off the A-slot barrier
+    static constexpr int kWBlocks = (I8 ? 2 : 1) * (BITS == 4 ? 1 : 2);  // packed blocks per k-step
+    static constexpr int kWBytes = I8 ? kWBlocks * kWeightBlockBytes : (BITS == 4 ? 5120 : 8192);
+    static constexpr int kWStages = I8 ? (BITS == 4 ? 6 : 4) : (BITS == 4 ? 9 : 6);
     static constexpr int kASlots = 8;                                    // tensor memory: 8 x 32 columns beside the accumulator
     static constexpr int kEarlySteps = kASlots - 2;                      // steps of the next tile dequantised before the epilogue is forced
     static constexpr int kWOffset = kXStages * kXBytes;
@@ -76,12 +79,14 @@ struct TaMaps {
 };
 
 // The packed body of a layer as a 2-D tensor of 64-byte rows; box = the block(s) of one 64-k step.
-inline bool w_tensor_map(const Layout& L, const uint8_t* blob, CUtensorMap* out)
+// i8: the integer form's box (128 k: two int4 blocks or four int8 blocks; per-channel schemes only).
+inline bool w_tensor_map(const Layout& L, const uint8_t* blob, CUtensorMap* out, bool i8 = false)
 {
     EncodeTiledFn enc = get_encode_tiled();
     if (!enc) return false;
+    if (i8 && L.grouped) return false;
     const int64_t rows = (int64_t)L.n_rsb * L.n_kc * (L.block_bytes / 64);
-    const int box_rows = L.bits == 4 ? L.block_bytes / 64 : 2 * (kWeightBlockBytes / 64);
+    const int box_rows = (i8 ? 2 : 1) * (L.bits == 4 ? L.block_bytes / 64 : 2 * (kWeightBlockBytes / 64));
     if (rows < box_rows || rows > 0x7FFFFFFFll) return false;
     const cuuint64_t gdim[2] = {64, (cuuint64_t)rows};
     const cuuint64_t gstr[1] = {64};
@@ -113,9 +118,39 @@ struct DequantRowTa {
     }
     // 32 consecutive k of the row (half h of the 64-k step) -> 16 registers = 16 columns of the row's TMEM lane.
     // Same arithmetic as unpack_int4_word / unpack_int8_words (exact integers, then one multiplication by the scale).
-    template <int BITS, bool GROUPED>
+    template <int BITS, bool GROUPED, bool I8 = false>
     __device__ __forceinline__ void convert(const unsigned char* wp, int h, uint32_t r[16]) const
     {
+        if (I8) {
+            // integer form: 64 consecutive k of the row (half h of the 128-k step) as the stored unsigned bytes
+            // (q + 8 or q + 128), 4 per column: no arithmetic, only the choice of nibbles / bytes and their order
+            if (BITS == 4) {
+                const unsigned char* rp = wp + h * kWeightBlockBytes;                        // packed block h of the step
+                const uint32_t sh = mask == 0x000F000Fu ? 0u : 4u;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 w = *reinterpret_cast<const uint4*>(rp + off[c]);
+                    // a word's nibbles of this row are slots 0, 2, 1, 3 (layout.h): k 8c .. 8c + 3 of a 32-k half per word pair
+                    r[2 * c + 0] = __byte_perm((w.x >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
+                    r[2 * c + 1] = __byte_perm((w.y >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
+                    r[8 + 2 * c + 0] = __byte_perm((w.z >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
+                    r[8 + 2 * c + 1] = __byte_perm((w.w >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
+                }
+            } else {
+                const uint32_t bsel = sel == 0x4140u ? 0x5410u : 0x7632u;                    // this row's byte pair of two words
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {                                                // blocks 2h, 2h + 1: 32 k each
+                    const unsigned char* rp = wp + (2 * h + b) * kWeightBlockBytes;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(rp + off[c]);
+                        r[8 * b + 2 * c + 0] = __byte_perm(w.x, w.y, bsel);
+                        r[8 * b + 2 * c + 1] = __byte_perm(w.z, w.w, bsel);
+                    }
+                }
+            }
+            return;
+        }
         if (BITS == 4) {
             const unsigned char* rp = wp + 8 * h;
 #pragma unroll
@@ -152,14 +187,18 @@ struct DequantRowTa {
 // the shared output tile (nothing is sent to memory); the up tile's epilogue multiplies what it finds there by the up
 // projection, every thread reading back the values it wrote itself, and only that product goes to y (paper Section
 // 3.6).  n_tiles then counts positions of ONE layer.
-template <int BITS, bool GROUPED, bool GATED = false>
+// I8 (per-channel schemes, not gated): maps.x describes int8 activations; the stored weight integers go to the A slots
+// unconverted, the MMAs are kind::i8 with an s32 accumulator, and the epilogue removes the storage offset (offset x the
+// sum of the token's quantised row) and applies both scales (paper Section 3.7, prefill stage).
+template <int BITS, bool GROUPED, bool GATED = false, bool I8 = false>
 __global__ void __launch_bounds__(kPairThreads, 1)
 gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
 {
-    using S = GemmTaSmem<BITS>;
+    static_assert(!I8 || (!GATED && !GROUPED), "the integer form: per-channel scales, plain output");
+    using S = GemmTaSmem<BITS, I8>;
     constexpr int NX = S::kXStages, NW = S::kWStages, NA = S::kASlots;
     constexpr int BN = 256;
-    constexpr int W_BOX_BYTES = BITS == 4 ? (GROUPED ? kWeightBlockBytes + kScaleBlockBytes : kWeightBlockBytes) : 2 * kWeightBlockBytes;
+    constexpr int W_BOX_BYTES = I8 ? S::kWBytes : BITS == 4 ? (GROUPED ? kWeightBlockBytes + kScaleBlockBytes : kWeightBlockBytes) : 2 * kWeightBlockBytes;
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -252,7 +291,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     if (warp == 0) {
         // ------------------------------------------------------------------ weight producer (each CTA feeds itself)
         if (lane == 0) {
-            constexpr int CHUNKS = BITS == 4 ? 1 : 2;                    // packed blocks per k-step
+            constexpr int CHUNKS = S::kWBlocks;                          // packed blocks per k-step
             int s = 0, issued = 0;
             uint32_t par = 1;
             bool ok = true;
@@ -295,7 +334,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                         if (!mbar_wait(aempty_bar(ao), (uint32_t)((g - NX) / NA) & 1, abort_flag, 0x180 + ao)) { ok = false; break; }
                     }
                     mbar_expect_tx(afull_bar(g % NA), S::kXBytes);
-                    tma_load_2d(xs_addr(s), &maps.x, (it_base + it) * kGemmKStep, m0, afull_bar(g % NA));
+                    tma_load_2d(xs_addr(s), &maps.x, (it_base + it) * S::kKStep, m0, afull_bar(g % NA));
                     if (++s == NX) s = 0;
                 }
             }
@@ -310,7 +349,8 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
         // registers); one elected lane issues.
         if (rank == 0) {
             // f16 x f16 -> f32, both operands K-major (A from tensor memory), M = 256 per pair, N = 256
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(((QL_TA_EXP & 256) ? 128 : BN) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            // (integer form: u8 weights x s8 activations -> s32)
+            const uint32_t idesc = (I8 ? (2u << 4) | (1u << 10) : (1u << 4)) | ((uint32_t)(((QL_TA_EXP & 256) ? 128 : BN) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
             const uint32_t b_lo0 = umma_desc_lo(xs_addr(0));
             int s = 0, a = 0;
             uint32_t apar = 0;
@@ -326,10 +366,11 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                     const uint32_t ta = tmem_base + (uint32_t)(kTaAccCols + a * kTaSlotCols);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kXBytes >> 4);
                     if (elect_one()) {
-                        umma_f16_pair_ta(tmem_base, ta, b_lo, idesc, it > 0 ? 1u : 0u);
 #pragma unroll
-                        for (int k4 = 1; k4 < 4; ++k4)                   // 16 k: 8 columns of A, 32 bytes of the B swizzle row
-                            umma_f16_pair_ta(tmem_base, ta + 8 * k4, b_lo + 2 * k4, idesc, 1u);
+                        for (int k4 = 0; k4 < 4; ++k4) {                 // 16 k (32 k of bytes): 8 columns of A, 32 bytes of the B swizzle row
+                            if (I8) umma_i8_pair_ta(tmem_base, ta + 8 * k4, b_lo + 2 * k4, idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                            else umma_f16_pair_ta(tmem_base, ta + 8 * k4, b_lo + 2 * k4, idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                        }
                         umma_commit_pair(aempty_bar(a));                 // frees the A slot and the x stage in both CTAs
                     }
                     __syncwarp();
@@ -447,7 +488,20 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                         __syncwarp();
                         if (lane == 0) mbar_arrive_remote(tempty_bar, 0);
                     }
-                    if (!(QL_TA_EXP & 2)) {
+                    if (I8) {
+                        // acc = sum (q + off) * xq: remove off * (sum of the token's quantised row), then both scales; the 32
+                        // tokens' scales and row sums come as whole lines (the arrays are padded to whole tiles)
+                        constexpr int OFF = BITS == 4 ? 8 : 128;
+#pragma unroll
+                        for (int v4 = 0; v4 < 8; ++v4) {
+                            const float4 f = __ldg(reinterpret_cast<const float4*>(p.a8_scale + m0 + cc) + v4);
+                            const int4 i = __ldg(reinterpret_cast<const int4*>(p.a8_rowsum + m0 + cc) + v4);
+                            orow[(cc + 4 * v4 + 0) * 128] = __float2half_rn(f.x * (scale * (float)((int)r[4 * v4 + 0] - OFF * i.x)));
+                            orow[(cc + 4 * v4 + 1) * 128] = __float2half_rn(f.y * (scale * (float)((int)r[4 * v4 + 1] - OFF * i.y)));
+                            orow[(cc + 4 * v4 + 2) * 128] = __float2half_rn(f.z * (scale * (float)((int)r[4 * v4 + 2] - OFF * i.z)));
+                            orow[(cc + 4 * v4 + 3) * 128] = __float2half_rn(f.w * (scale * (float)((int)r[4 * v4 + 3] - OFF * i.w)));
+                        }
+                    } else if (!(QL_TA_EXP & 2)) {
 #pragma unroll
                         for (int q = 0; q < 32; ++q) {
                             float v = __uint_as_float(r[q]) * scale;
@@ -500,7 +554,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             }
             uint32_t r[16];
             if (!mbar_wait(wfull_bar(s), wpar, abort_flag, 0x400 + s)) { ok = false; break; }
-            if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED>(wpk_ptr(s), half, r);
+            if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED, I8>(wpk_ptr(s), half, r);
             else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = 0;
@@ -545,16 +599,19 @@ inline int gemm_pair_ta_split(int tiles, int n_ksteps, int num_sms, bool have_sc
 
 // act < 0: the plain form.  act >= 0: the gated form, set = {gate, up} of equal shape, y[0] the output.
 // scratch / counters: the device's shared fp32 scratch and arrival counters for the K-split case (null: no split).
-template <int BITS, bool GROUPED, bool GATED = false>
+// a8_scale != nullptr: the integer form; x is then the int8 activations, a8_scale / a8_rowsum their per-token arrays, and
+// set.wmap the integer form's weight maps (boxes of 128 k).
+template <int BITS, bool GROUPED, bool GATED = false, bool I8 = false>
 ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms, int act = -1,
-                              float* scratch = nullptr, unsigned int* counters = nullptr)
+                              float* scratch = nullptr, unsigned int* counters = nullptr,
+                              const float* a8_scale = nullptr, const int32_t* a8_rowsum = nullptr)
 {
-    using S = GemmTaSmem<BITS>;
+    using S = GemmTaSmem<BITS, I8>;
     const Layout& L = *set.L[0];
     TaMaps maps;
-    if (!x_tensor_map(x, L.K, M, 128, &maps.x)) return QL_ERR_CUDA;
+    if (!x_tensor_map(x, L.K, M, 128, &maps.x, I8 ? 1 : 2)) return QL_ERR_CUDA;
     for (int i = 0; i < kGemmMaxGroup; ++i) maps.w[i] = *set.wmap[i < set.n ? i : 0];
-    auto kern = gemm_pair_ta_kernel<BITS, GROUPED, GATED>;
+    auto kern = gemm_pair_ta_kernel<BITS, GROUPED, GATED, I8>;
     static std::atomic<bool> attr_set[64];
     if (device >= 0 && device < 64 && !attr_set[device]) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) {
@@ -581,10 +638,11 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
     if (GATED) n_rsb = L.n_rsb;                                          // work units count positions of one layer
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
-    prm.n_ksteps = (L.K + kGemmKStep - 1) / kGemmKStep;
+    prm.n_ksteps = (L.K + S::kKStep - 1) / S::kKStep;
+    prm.a8_scale = a8_scale; prm.a8_rowsum = a8_rowsum;
     prm.n_rsb = n_rsb;
     prm.n_tiles = (n_rsb / 2) * ((M + 255) / 256);
-    prm.split = GATED ? 1 : gemm_pair_ta_split(prm.n_tiles, prm.n_ksteps, num_sms, scratch && counters);
+    prm.split = (GATED || I8) ? 1 : gemm_pair_ta_split(prm.n_tiles, prm.n_ksteps, num_sms, scratch && counters);
     prm.scratch = scratch;
     prm.counters = counters;
     prm.n_whole = prm.n_tiles;
@@ -644,6 +702,22 @@ inline ql_status gemm_pair_ta_forward_gated(const GemmPairLayers& set, const voi
     if (L.bits == 8) return gemm_pair_ta_launch<8, false, true>(set, x, M, st, device, pdl, num_sms, act);
     if (L.grouped) return gemm_pair_ta_launch<4, true, true>(set, x, M, st, device, pdl, num_sms, act);
     return gemm_pair_ta_launch<4, false, true>(set, x, M, st, device, pdl, num_sms, act);
+}
+
+// Integer form (per-channel schemes, K a multiple of 128): xq int8 [M, K] with per-token scale and row sum; set.wmap
+// holds the integer form's weight maps.  No K split: launches with fewer tiles than half the CTA pairs stay on the
+// shared-memory kernel.
+inline bool gemm_pair_ta_i8_applicable(const GemmPairLayers& set, int M, int num_sms)
+{
+    if (!gemm_config().ta || M <= 128 || !set.wmap[0]) return false;
+    return set.L[0]->n_rsb / 2 * ((M + 255) / 256) * 2 > num_sms / 2;
+}
+inline ql_status gemm_pair_ta_forward_i8(const GemmPairLayers& set, const void* xq, const float* scale, const int32_t* rowsum, int M,
+                                         cudaStream_t st, int device, bool pdl, int num_sms)
+{
+    const Layout& L = *set.L[0];
+    if (L.bits == 8) return gemm_pair_ta_launch<8, false, false, true>(set, xq, M, st, device, pdl, num_sms, -1, nullptr, nullptr, scale, rowsum);
+    return gemm_pair_ta_launch<4, false, false, true>(set, xq, M, st, device, pdl, num_sms, -1, nullptr, nullptr, scale, rowsum);
 }
 
 // The CTA-pair prefill call: the tensor-memory form where it applies, else the shared-memory form.

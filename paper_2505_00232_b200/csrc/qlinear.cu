@@ -130,7 +130,8 @@ struct qlinear_s {
     bool use_stream;
     int stream_P, stream_stages;
     CUtensorMap wmap;          // the packed body as rows of 64 bytes (prefill kernel with the weights in tensor memory)
-    bool wmap_ok;
+    CUtensorMap wmap_i8;       // the same with the integer form's box (128 k per step)
+    bool wmap_ok, wmap_i8_ok;
     DeviceState* dev;
 };
 
@@ -463,6 +464,7 @@ extern "C" ql_status qlinear_create(const qlinear_desc* d, const void* packed_de
     h->pdl = cfg.pdl;
     h->n_rb = (L.N + kRbRows - 1) / kRbRows;
     h->wmap_ok = w_tensor_map(L, h->blob, &h->wmap);
+    h->wmap_i8_ok = !L.grouped && (L.K % 128) == 0 && w_tensor_map(L, h->blob, &h->wmap_i8, true);
     for (int M = 1; M <= 8; ++M) {
         h->gemv[M] = plan_gemv(L, h->n_rb, M, sms);
         if (h->gemv[M].grid <= 0 && M <= h->gemv_max_m) { delete h; return QL_ERR_UNSUPPORTED; }   // no decode plan fits this shape
@@ -627,7 +629,8 @@ extern "C" ql_status qlinear_forward_a8(qlinear_t h, const void* x, void* y, int
         quantize_activations_kernel<<<M, 256, 0, st>>>(static_cast<const __half*>(x), xq, sx, rs, M, L.K);
         if (cudaGetLastError() != cudaSuccess) return QL_ERR_CUDA;
         GemmPairLayers set{};
-        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y;
+        set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y; set.wmap[0] = h->wmap_i8_ok ? &h->wmap_i8 : nullptr;
+        if (gemm_pair_ta_i8_applicable(set, M, h->num_sms)) return gemm_pair_ta_forward_i8(set, xq, sx, rs, M, st, h->device, h->pdl, h->num_sms);
         return gemm_pair_forward_i8(set, xq, sx, rs, M, st, h->device, h->pdl, h->num_sms);
     }
     const GemvPlan pl = plan_gemv(L, h->n_rb, M, h->num_sms, false, true);
