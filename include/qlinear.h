@@ -28,9 +28,11 @@
  *
  * Device memory.  The caller owns the packed weights, x and y.  The library
  * owns one small set of buffers PER DEVICE, allocated when the first handle on
- * that device is created and kept until the process exits: about 19 MB of fp32
- * partial tiles plus counters for the K-split prefill case, and one word of
- * pinned host memory through which kernels report an expired wait.  A handle
+ * that device is created and kept until the process exits: 40 MB of scratch
+ * (fp32 partial tiles of the K-split prefill case, the int8 activations of the
+ * integer prefill form, the two projections of the unfused gating route) plus
+ * arrival counters, and one word of pinned host memory through which kernels
+ * report an expired wait.  A handle
  * itself owns host memory only.
  *
  * Environment.  Every QLINEAR_* variable is read once per process, at the
