@@ -106,3 +106,37 @@ def test_guard_band_around_y(P, torch):
     y64, A, _ = O.linear(x, q, s, group)
     ok, rel, worst = O.check_against(y, y64, A)
     assert ok, f"rel_l2={rel:.3e} worst={worst:.3e}"
+
+
+def test_dependent_launches_back_to_back(P, torch):
+    """A chain y1 = L1(x), y2 = L2(y1), y3 = L3(y2) launched without any host synchronisation (each kernel releases the
+    next one early and the next one may already run its set-up): same bits as the chain with a synchronise after every
+    launch, on every repetition, with the buffers reused."""
+    M, D = 1500, 4864                                                    # 19 row-super-block pairs x 6 token blocks = 114 tiles
+    lins = []
+    for i, (bits, group) in enumerate([(4, 32), (8, 0), (4, 0)]):
+        q, s, _ = case(900 + i, 8, D, D, bits, group)
+        desc = P.Desc(D, D, bits, group)
+        lins.append(P.QLinear(desc, torch.from_numpy(P.qlinear_pack(desc, q, (s.astype(np.float32) / 16).astype(np.float16))).cuda()))
+    x = torch.from_numpy(case(77, M, D, D, 4, 32)[2]).cuda()
+    bufs = [torch.empty((M, D), dtype=torch.float16, device="cuda") for _ in range(3)]
+
+    def chain(sync):
+        src = x
+        for lin, dst in zip(lins, bufs):
+            lin.forward_raw(src.data_ptr(), dst.data_ptr(), M)
+            if sync:
+                torch.cuda.synchronize()
+            src = dst
+        torch.cuda.synchronize()
+        return [b.clone() for b in bufs]
+
+    ref = chain(True)
+    assert all(torch.isfinite(r.float()).all() for r in ref)
+    for _ in range(5):
+        for b in bufs:
+            b.fill_(float("nan"))
+        got = chain(False)
+        for r, g in zip(ref, got):
+            assert torch.equal(r.view(torch.int16), g.view(torch.int16))
+    assert lins[0].device_status() == (0, 0)
