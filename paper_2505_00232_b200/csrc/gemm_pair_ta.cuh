@@ -99,6 +99,26 @@ inline bool w_tensor_map(const Layout& L, const uint8_t* blob, CUtensorMap* out,
 
 // Per-thread constants of a dequantise warp: the thread's tile row is TMEM lane 32 * quarter + lane, i.e. row-block
 // 2 * quarter + lane / 16, lane-row g = lane % 8, upper half (rows g + 8) for lanes 8..15 and 24..31.
+// Shared-memory loads through 32-bit shared-window addresses (a generic pointer costs 64-bit address arithmetic per load).
+__device__ __forceinline__ uint2 lds_u64(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint4 lds_u128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t addr)
+{
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return v;
+}
+
 struct DequantRowTa {
     int off[4];                  // byte offset, inside the packed block, of piece c of the row's 64-byte line (64-byte swizzle:
                                  // piece c sits at position c ^ ((line / 2) & 3))
@@ -119,17 +139,17 @@ struct DequantRowTa {
     // 32 consecutive k of the row (half h of the 64-k step) -> 16 registers = 16 columns of the row's TMEM lane.
     // Same arithmetic as unpack_int4_word / unpack_int8_words (exact integers, then one multiplication by the scale).
     template <int BITS, bool GROUPED, bool I8 = false>
-    __device__ __forceinline__ void convert(const unsigned char* wp, int h, uint32_t r[16]) const
+    __device__ __forceinline__ void convert(uint32_t wp, int h, uint32_t r[16]) const   // wp: shared-window address of the stage
     {
         if (I8) {
             // integer form: 64 consecutive k of the row (half h of the 128-k step) as the stored unsigned bytes
             // (q + 8 or q + 128), 4 per column: no arithmetic, only the choice of nibbles / bytes and their order
             if (BITS == 4) {
-                const unsigned char* rp = wp + h * kWeightBlockBytes;                        // packed block h of the step
+                const uint32_t rp = wp + h * kWeightBlockBytes;                              // packed block h of the step
                 const uint32_t sh = mask == 0x000F000Fu ? 0u : 4u;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint4 w = *reinterpret_cast<const uint4*>(rp + off[c]);
+                    const uint4 w = lds_u128(rp + off[c]);
                     // a word's nibbles of this row are slots 0, 2, 1, 3 (layout.h): k 8c .. 8c + 3 of a 32-k half per word pair
                     r[2 * c + 0] = __byte_perm((w.x >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
                     r[2 * c + 1] = __byte_perm((w.y >> sh) & 0x0F0F0F0Fu, 0, 0x3120);
@@ -140,10 +160,10 @@ struct DequantRowTa {
                 const uint32_t bsel = sel == 0x4140u ? 0x5410u : 0x7632u;                    // this row's byte pair of two words
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {                                                // blocks 2h, 2h + 1: 32 k each
-                    const unsigned char* rp = wp + (2 * h + b) * kWeightBlockBytes;
+                    const uint32_t rp = wp + (2 * h + b) * kWeightBlockBytes;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const uint4 w = *reinterpret_cast<const uint4*>(rp + off[c]);
+                        const uint4 w = lds_u128(rp + off[c]);
                         r[8 * b + 2 * c + 0] = __byte_perm(w.x, w.y, bsel);
                         r[8 * b + 2 * c + 1] = __byte_perm(w.z, w.w, bsel);
                     }
@@ -152,26 +172,26 @@ struct DequantRowTa {
             return;
         }
         if (BITS == 4) {
-            const unsigned char* rp = wp + 8 * h;
+            const uint32_t rp = wp + 8 * h;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const uint2 w = *reinterpret_cast<const uint2*>(rp + off[c]);
+                const uint2 w = lds_u64(rp + off[c]);
                 r[4 * c + 0] = h2_fma(lop3_and_or(w.x, mask, 0x64006400u), mul, add);        // k 8c + 0, 1
                 r[4 * c + 1] = h2_fma(lop3_and_or(w.x >> 8, mask, 0x64006400u), mul, add);   // k 8c + 2, 3
                 r[4 * c + 2] = h2_fma(lop3_and_or(w.y, mask, 0x64006400u), mul, add);        // k 8c + 4, 5
                 r[4 * c + 3] = h2_fma(lop3_and_or(w.y >> 8, mask, 0x64006400u), mul, add);   // k 8c + 6, 7
             }
             if (GROUPED) {
-                const uint32_t s = *reinterpret_cast<const uint16_t*>(wp + s_off + 2 * h);
+                const uint32_t s = lds_u16(wp + s_off + 2 * h);
                 const uint32_t s2 = s | (s << 16);
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = h2_mul(r[i], s2);
             }
         } else {
-            const unsigned char* rp = wp + h * kWeightBlockBytes;                            // chunk h of the step
+            const uint32_t rp = wp + h * kWeightBlockBytes;                                  // chunk h of the step
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const uint4 w = *reinterpret_cast<const uint4*>(rp + off[c]);
+                const uint4 w = lds_u128(rp + off[c]);
                 r[4 * c + 0] = h2_sub(__byte_perm(w.x, 0x64646464u, sel), 0x64806480u);
                 r[4 * c + 1] = h2_sub(__byte_perm(w.y, 0x64646464u, sel), 0x64806480u);
                 r[4 * c + 2] = h2_sub(__byte_perm(w.z, 0x64646464u, sel), 0x64806480u);
@@ -204,7 +224,6 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
     unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
     auto xs_addr = [&](int s) { return base + s * S::kXBytes; };
     auto wpk_addr = [&](int s) { return base + S::kWOffset + s * S::kWBytes; };
-    auto wpk_ptr = [&](int s) { return base_ptr + S::kWOffset + s * S::kWBytes; };
     const uint32_t bar0 = base + S::kBarOffset;
     // (barrier slots 0 .. NX-1 are unused: the x tile of a step completes on the step's afull barrier)
     auto wfull_bar = [&](int s) { return bar0 + 8 * (NX + s); };         // local: this CTA's packed block landed
@@ -554,7 +573,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             }
             uint32_t r[16];
             if (!mbar_wait(wfull_bar(s), wpar, abort_flag, 0x400 + s)) { ok = false; break; }
-            if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED, I8>(wpk_ptr(s), half, r);
+            if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED, I8>(wpk_addr(s), half, r);
             else {
 #pragma unroll
                 for (int i = 0; i < 16; ++i) r[i] = 0;
