@@ -26,7 +26,7 @@
 //
 // What bounds it (measured): not the tensor pipe (halving the MMA width changes nothing) but the instruction stream
 // of the dequantise warps and of the polling threads around them, which is why every warp loops over its own steps
-// only and only the MMA issuer polls.
+// only and no thread polls in the main loop.
 //
 // Protocol between the two CTAs: own loads only; the leader issues; commits are multicast to both CTAs; the peer relays
 // "slot ready" (see the relay below).
@@ -380,7 +380,8 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                 tc_fence_after();
                 for (int it = 0; it < n_steps; ++it) {
                     // both CTAs' A slots written and both x tiles landed (8 local warps, the local x tile, the peer's relay)
-                    if (!mbar_wait_hot(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
+                    // (the dequantise warps run ahead, so the phase is normally complete already: test, else suspend)
+                    if (!mbar_wait(afull_bar(a), apar, abort_flag, 0x300 + a)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t ta = tmem_base + (uint32_t)(kTaAccCols + a * kTaSlotCols);
                     const uint32_t b_lo = b_lo0 + (uint32_t)s * (S::kXBytes >> 4);
