@@ -690,14 +690,17 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
     return QL_OK;
 }
 
+// Any M the prefill path sees (tokens beyond M are zero-filled by TMA and never stored): below 129 tokens the tile is
+// mostly padding, but the launch is bound by streaming and dequantising the weights, which this kernel spreads over
+// the whole GPU (K split), not by the MMAs.
 inline bool gemm_pair_ta_applicable(const GemmPairLayers& set, int M, int num_sms, bool gated = false)
 {
-    if (!gemm_config().ta || M <= 128) return false;
+    if (!gemm_config().ta || !gemm_config().pair) return false;
     for (int i = 0; i < set.n; ++i)
-        if (!set.wmap[i]) return false;
+        if (!set.wmap[i] || (set.L[i]->n_rsb % 2)) return false;
     // the gated form needs a whole number of positions per round of the grid's clusters to be worth it; the plain form
     // takes every launch (few tiles: fewer clusters, or a K split through the device scratch)
-    return !gated || (set.L[0]->n_rsb / 2) * ((M + 255) / 256) >= num_sms / 2;
+    return !gated || (M > 128 && (set.L[0]->n_rsb / 2) * ((M + 255) / 256) >= num_sms / 2);
 }
 
 inline ql_status gemm_pair_ta_forward(const GemmPairLayers& set, const void* x, int M, cudaStream_t st, int device, bool pdl, int num_sms,
@@ -745,6 +748,8 @@ inline ql_status gemm_pair_forward_auto(const GemmPairLayers& set, const void* x
                                         int device, bool pdl, int num_sms, float* scratch, unsigned int* counters)
 {
     if (gemm_pair_ta_applicable(set, M, num_sms)) return gemm_pair_ta_forward(set, x, M, st, device, pdl, num_sms, scratch, counters);
+    for (int i = 0; i < set.n; ++i)
+        if (!gemm_pair_applicable(*set.L[i], M)) return QL_ERR_UNSUPPORTED;
     return gemm_pair_forward(set, x, M, st, device, pdl, num_sms, scratch, counters);
 }
 

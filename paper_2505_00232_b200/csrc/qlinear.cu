@@ -507,10 +507,11 @@ extern "C" ql_status qlinear_forward(qlinear_t h, const void* x, void* y, int32_
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (M <= h->gemv_max_m) return h->use_stream ? forward_gemv_stream(h, x, y, M, st) : forward_gemv(&h, 1, x, &y, M, st);
-    if (gemm_pair_applicable(h->L, M)) {
+    {
         GemmPairLayers set{};
         set.n = 1; set.L[0] = &h->L; set.blob[0] = h->blob; set.y[0] = y; set.wmap[0] = h->wmap_ok ? &h->wmap : nullptr;
-        return gemm_pair_forward_auto(set, x, M, st, h->device, h->pdl, h->num_sms, h->dev->gemm_scratch, h->dev->gemm_counters);
+        const ql_status s = gemm_pair_forward_auto(set, x, M, st, h->device, h->pdl, h->num_sms, h->dev->gemm_scratch, h->dev->gemm_counters);
+        if (s != QL_ERR_UNSUPPORTED) return s;                           // (an odd number of row super-blocks: the single-CTA kernel)
     }
     return gemm_forward(h->L, h->blob, x, y, M, st, h->device, h->pdl, h->num_sms);
 }
@@ -534,7 +535,7 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
     }
     if (n > 1 && M > hs[0]->gemv_max_m) {                                // prefill: one launch of the CTA-pair kernel
         bool pair_ok = true;
-        for (int i = 0; i < n; ++i) pair_ok = pair_ok && gemm_pair_applicable(hs[i]->L, M);
+        for (int i = 0; i < n; ++i) pair_ok = pair_ok && (hs[i]->L.n_rsb % 2) == 0 && (gemm_pair_applicable(hs[i]->L, M) || (hs[i]->wmap_ok && gemm_config().ta));
         if (pair_ok) {
             DeviceGuard guard(hs[0]->device);
             if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
@@ -544,8 +545,9 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
                 set.L[i] = &hs[i]->L; set.blob[i] = hs[i]->blob; set.y[i] = ys[i];
                 set.wmap[i] = hs[i]->wmap_ok ? &hs[i]->wmap : nullptr;
             }
-            return gemm_pair_forward_auto(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
-                                     hs[0]->dev->gemm_scratch, hs[0]->dev->gemm_counters);
+            const ql_status s = gemm_pair_forward_auto(set, x, M, static_cast<cudaStream_t>(stream), hs[0]->device, hs[0]->pdl, hs[0]->num_sms,
+                                                       hs[0]->dev->gemm_scratch, hs[0]->dev->gemm_counters);
+            if (s != QL_ERR_UNSUPPORTED) return s;
         }
     }
     for (int i = 0; i < n; ++i) {
