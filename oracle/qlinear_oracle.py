@@ -24,8 +24,9 @@ Parity pins: tests/test_oracle_pins.py (worked examples stored under
 tests/golden/, brute force over all byte values, one-hot / zero / closed-form
 cases, power-of-two and negation invariants, a double-rounding trap) and
 tests/test_oracle_pins_next.py for the three extensions further down (fused
-gating, Section 3.6; int8 activation quantisation, Section 3.7; the KV cache as
-weights, Section 3.8).  No function here is unpinned.
+gating and residual + RMS normalisation, Section 3.6; int8 activation
+quantisation, Section 3.7; the KV cache as weights, Section 3.8).  No function
+here is unpinned.
 """
 from __future__ import annotations
 
@@ -252,6 +253,37 @@ def kv_scores(qry, k_q, k_s):
 def kv_output(prob, v_q, v_s):
     """out64 [R, d_h] = prob [R, T] . V, V cache v_q int8 [d_h, T] (O = d_h, I = T), v_s fp16 [d_h]."""
     return linear(prob, v_q, v_s, 0)
+
+
+# ----------------------------------------------------------------------------- residual + RMS normalisation (paper Section 3.6)
+# The paper's second fusion example merges "residual connection and element-wise operations with a manually optimized
+# RMS normalization operator": the operator that produces the linear layer's input.  The paper gives no formulas; the
+# readings taken (recorded in the design notes) are the ones the paper's models use:
+#   h[m,k]  = x[m,k] + r[m,k]                                   residual connection (the sum of two fp16 values, exact)
+#   ms[m]   = (1/K) * sum_k h[m,k]^2                            mean square over the hidden dimension
+#   y[m,k]  = h[m,k] / sqrt(ms[m] + eps) * (offset + g[k])      RMS normalisation with its element-wise scale
+#             (offset = 0: Llama; offset = 1: Gemma stores the scale as g - 1)
+# The normalisation is computed from the UNROUNDED sum h (a merged operator has it in registers); the operator also
+# returns fp16(h), the residual stream for the next block.  Everything in fp64 here, one rounding to fp16 per output.
+def residual_rmsnorm(x, r, g, eps: float, offset: float = 0.0):
+    """x, r fp16 [M, K] (r may be None: no residual), g fp16 [K] -> (h64, h16, y64, y16)."""
+    h = np.asarray(x, dtype=np.float16).astype(np.float64)
+    if r is not None:
+        h = h + np.asarray(r, dtype=np.float16).astype(np.float64)
+    ms = np.mean(h * h, axis=1, keepdims=True)
+    y = h / np.sqrt(ms + float(eps)) * (float(offset) + np.asarray(g, dtype=np.float16).astype(np.float64))[None, :]
+    with np.errstate(over="ignore"):
+        return h, h.astype(np.float16), y, y.astype(np.float16)
+
+
+def residual_rmsnorm_bound(h64, y64, K: int):
+    """Acceptance bounds (|dh|, |dy|) for an fp32 implementation: h is exact before its rounding (2^-11 relative, or
+    2^-25 absolute among the fp16 subnormals); y carries that rounding plus the fp32 arithmetic: a sum of K squares
+    kept in at least 128 partial sums that are then added pairwise (K / 128 + 7 additions deep), the square root, the
+    division and two multiplications, half an fp32 ulp (2^-24) each, first order."""
+    bh = 2.0 ** -11 * np.abs(h64) + 2.0 ** -25
+    by = (2.0 ** -11 + (K / 128.0 + 7 + 5) * 2.0 ** -24) * np.abs(y64) + 2.0 ** -25
+    return bh, by
 
 
 # ----------------------------------------------------------------------------- C oracle

@@ -226,3 +226,87 @@ def test_kv_attention_matches_a_plain_float_attention_closely_and_exactly_on_the
     sc64, _, out64, _ = O.kv_attention(qry, kg, vg, pg)
     np.testing.assert_allclose(sc64, qry.astype(np.float64) @ kg.astype(np.float64).T, rtol=1e-13, atol=1e-12)
     np.testing.assert_allclose(out64, pg.astype(np.float64) @ vg.astype(np.float64), rtol=1e-13, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- residual + RMS normalisation
+def test_example_I_residual_rmsnorm(golden):
+    e = golden["I_residual_rmsnorm"]
+    h64, h16, y64, y16 = O.residual_rmsnorm(np.array(e["x"], np.float16), np.array(e["r"], np.float16),
+                                            np.array(e["g"], np.float16), e["eps"], e["offset"])
+    assert (h64 == np.array(e["h64"])).all() and (y64 == np.array(e["y64"])).all()       # exact: powers of two throughout
+    assert (h16 == h64).all() and (y16 == y64).all()
+
+
+def test_rmsnorm_against_plain_loops_and_the_library_routine():
+    import torch
+    rng = np.random.default_rng(5)
+    M, K = 7, 96
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    r = (3 * rng.standard_normal((M, K))).astype(np.float16)
+    g = rng.standard_normal(K).astype(np.float16)
+    eps, off = 1e-5, 1.0
+    h64, _, y64, _ = O.residual_rmsnorm(x, r, g, eps, off)
+    for m in range(M):                                                   # the definition written out with Python floats
+        h = [float(x[m, k]) + float(r[m, k]) for k in range(K)]
+        ms = math.fsum(v * v for v in h) / K
+        for k in range(K):
+            assert h64[m, k] == h[k]
+            assert y64[m, k] == pytest.approx(h[k] / math.sqrt(ms + eps) * (off + float(g[k])), rel=1e-14, abs=0)
+    # special case the library has: no residual, offset 0
+    _, _, y0, _ = O.residual_rmsnorm(x, None, g, eps, 0.0)
+    ref = torch.nn.functional.rms_norm(torch.from_numpy(x.astype(np.float64)), (K,), torch.from_numpy(g.astype(np.float64)), eps)
+    np.testing.assert_allclose(y0, ref.numpy(), rtol=1e-13, atol=0)
+
+
+def test_rmsnorm_invariants():
+    rng = np.random.default_rng(6)
+    M, K = 5, 64
+    x = rng.standard_normal((M, K)).astype(np.float16)
+    r = rng.standard_normal((M, K)).astype(np.float16)
+    g = (1 + rng.standard_normal(K) / 4).astype(np.float16)
+    # without eps the output does not change when the input is scaled (power of two: exact); the sign follows
+    _, _, y1, _ = O.residual_rmsnorm(x, r, g, 0.0)
+    _, _, y2, _ = O.residual_rmsnorm((x * np.float16(-4)).astype(np.float16), (r * np.float16(-4)).astype(np.float16), g, 0.0)
+    np.testing.assert_allclose(y2, -y1, rtol=1e-15, atol=0)
+    # mean of (y / scale)^2 is ms / (ms + eps)
+    eps = 0.37
+    h64, _, y, _ = O.residual_rmsnorm(x, r, g, eps)
+    ms = (h64 ** 2).mean(axis=1)
+    np.testing.assert_allclose(((y / g.astype(np.float64)) ** 2).mean(axis=1), ms / (ms + eps), rtol=1e-13)
+    # the residual branch is a plain sum: the two inputs commute, and no residual is a residual of zeros
+    a = O.residual_rmsnorm(x, r, g, eps, 1.0)
+    b = O.residual_rmsnorm(r, x, g, eps, 1.0)
+    assert all((u == v).all() for u, v in zip(a, b))
+    c = O.residual_rmsnorm(x, None, g, eps)
+    d = O.residual_rmsnorm(x, np.zeros_like(x), g, eps)
+    assert all((u == v).all() for u, v in zip(c, d))
+    # a constant row comes out as +-scale (eps = 0), whatever the constant
+    _, _, yc, _ = O.residual_rmsnorm(np.full((1, K), -3.0, np.float16), None, g, 0.0)
+    np.testing.assert_allclose(yc[0], -g.astype(np.float64), rtol=1e-15)
+
+
+def test_rmsnorm_bound_holds_for_an_fp32_emulation():
+    rng = np.random.default_rng(8)
+    M, K = 16, 4096
+    x = (2 * rng.standard_normal((M, K))).astype(np.float16)
+    r = (8 * rng.standard_normal((M, K))).astype(np.float16)
+    g = rng.standard_normal(K).astype(np.float16)
+    eps = 1e-6
+    h64, _, y64, _ = O.residual_rmsnorm(x, r, g, eps, 0.0)
+    bh, by = O.residual_rmsnorm_bound(h64, y64, K)
+    h32 = x.astype(np.float32) + r.astype(np.float32)
+    part = np.zeros((M, 128), np.float32)                                # 128 partial sums, then pairwise
+    for k0 in range(0, K, 128):
+        part = (part + h32[:, k0:k0 + 128] * h32[:, k0:k0 + 128]).astype(np.float32)
+    while part.shape[1] > 1:
+        part = (part[:, 0::2] + part[:, 1::2]).astype(np.float32)
+    ss = part[:, 0]
+    rstd = (np.float32(1) / np.sqrt((ss / np.float32(K) + np.float32(eps)).astype(np.float32))).astype(np.float32)
+    y32 = ((h32 * rstd[:, None]).astype(np.float32) * g.astype(np.float32)[None, :]).astype(np.float32)
+    assert (np.abs(h32.astype(np.float16).astype(np.float64) - h64) <= bh).all()
+    assert (np.abs(y32.astype(np.float16).astype(np.float64) - y64) <= by).all()
+    # and a wrong divisor (mean over K - 1) is caught where 1 / (2 K) exceeds an fp16 rounding
+    K2 = 64
+    h2, _, y2, _ = O.residual_rmsnorm(x[:, :K2], r[:, :K2], g[:K2], eps, 0.0)
+    _, by2 = O.residual_rmsnorm_bound(h2, y2, K2)
+    assert (np.abs(y2 * np.sqrt(K2 / (K2 - 1.0)) - y2) > by2).any()
