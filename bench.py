@@ -632,6 +632,7 @@ def main():
             if not args.no_configs:
                 line["configs"] += prefill_configs(torch, device, peaks, sidx, line)
                 line["fused_gating"] = gated_record(torch, device, peaks, sidx, ls)
+                line["residual_rmsnorm"] = norm_record(torch, device, peaks, sidx)
                 line["int8_activations"] = a8_record(torch, device, peaks, sidx)
         # ---- CPU oracle beside it (bounded sample)
         if not args.no_cpu_baseline:
@@ -671,6 +672,28 @@ def prefill_sub(torch, device, peaks, steps, sidx, blobs):
            "roofline": prefill_roofline(torch, ls, w, M, peaks, sidx)}
     del ls
     torch.cuda.empty_cache()
+    return out
+
+
+def norm_record(torch, device, peaks, sidx):
+    """Residual connection + RMS normalisation (paper Section 3.6), the operator that produces the linear layer's
+    input, at the Llama width: prefill (M = 2048; 8 rotated buffer sets = 537 MB, past L2) and one decode token."""
+    import paper_2505_00232_b200 as P
+    K, out = 4096, {"K": 4096, "bytes_per_token": 4 * 4096 * 2}
+    rng = np.random.default_rng(3)
+    g = torch.from_numpy((rng.standard_normal(K) / 4).astype(np.float16)).to(device)
+    for stage, M, sets in (("prefill", 2048, 8), ("decode", 1, 64)):
+        xs = [torch.from_numpy(rng.standard_normal((M, K)).astype(np.float16)).to(device) for _ in range(sets)]
+        rs = [torch.from_numpy(rng.standard_normal((M, K)).astype(np.float16)).to(device) for _ in range(sets)]
+        hs = [torch.empty_like(xs[0]) for _ in range(sets)]
+        ys = [torch.empty_like(xs[0]) for _ in range(sets)]
+        graph = capture_graph(torch, lambda i: P.qlinear_residual_rmsnorm(xs[i], rs[i], g, 1e-5, 0.0, h_out=hs[i], y_out=ys[i]), sets)
+        for _ in range(3):
+            graph.replay()
+        ms, repeats, clocks = timed_region(torch, graph.replay, sets, sidx, 0.25)
+        us = ms * 1e3 / (repeats * sets)
+        gbs = 4 * M * K * 2 / 1e3 / us
+        out[stage] = {"M": M, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
     return out
 
 

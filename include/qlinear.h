@@ -225,6 +225,21 @@ ql_status qlinear_kv_output(qlinear_t h_v, const void* prob_dev, const void* v_s
  * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, n < 0), QL_ERR_CUDA (launch failure). */
 ql_status qlinear_embed(qlinear_t h, const int32_t* ids_dev, int32_t n, void* y_dev, void* cuda_stream);
 
+/* Residual connection + RMS normalisation: the operator that PRODUCES the linear layer's input (paper Section 3.6,
+ * second fusion example: the residual connection and the element-wise operations merged with the RMS normalisation
+ * operator).  Per token m (row of K values):
+ *     h[m,k] = x[m,k] + residual[m,k]                               (fp32; residual may be NULL: h = x)
+ *     y[m,k] = h[m,k] / sqrt(mean_k h[m,k]^2 + eps) * (gamma_offset + gamma[k])
+ * h_out (may be NULL) receives fp16(h), the residual stream of the next block; y_out receives fp16(y).  The paper gives
+ * no formulas; these are the ones of the models it runs (gamma_offset = 0: Llama; 1: Gemma, which stores gamma - 1).
+ * x_dev, residual_dev, h_out_dev, y_out_dev: fp16 [M, K] row-major, device memory of `device`, 16-byte aligned;
+ * gamma_dev: fp16 [K].  K a multiple of 8; M >= 0 (0: nothing is done); eps >= 0.  h_out_dev may be x_dev or
+ * residual_dev (in place), y_out_dev may be x_dev; h_out_dev and y_out_dev must differ.  No handle, no library-owned
+ * memory; asynchronous on cuda_stream.  Returns QL_ERR_INVALID_ARG for null / misaligned pointers or a bad shape,
+ * QL_ERR_CUDA if the launch fails. */
+ql_status qlinear_residual_rmsnorm(const void* x_dev, const void* residual_dev, const void* gamma_dev, float eps, float gamma_offset,
+                                   void* h_out_dev, void* y_out_dev, int32_t M, int32_t K, int32_t device, void* cuda_stream);
+
 /* The kernel qlinear_forward uses for M tokens on this handle (0 if h is NULL or M < 1). */
 int32_t qlinear_path_for(qlinear_t h, int32_t M);
 

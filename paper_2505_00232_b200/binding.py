@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -76,6 +76,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_kv_output.restype = ctypes.c_int
     lib.qlinear_embed.argtypes = [vp, vp, ctypes.c_int32, vp, vp]
     lib.qlinear_embed.restype = ctypes.c_int
+    lib.qlinear_residual_rmsnorm.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp, i32, i32, ctypes.c_int, vp]
+    lib.qlinear_residual_rmsnorm.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
     lib.qlinear_debug_expire_wait.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -238,6 +240,30 @@ def qlinear_quantize_activations(x, stream=None):
     _check(lib.qlinear_quantize_activations(ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(xq.data_ptr()), ctypes.c_void_p(scale.data_ptr()),
                                             M, K, x.device.index or 0, _stream_ptr(stream)), "qlinear_quantize_activations")
     return xq, scale
+
+
+def qlinear_residual_rmsnorm(x, residual, gamma, eps: float, gamma_offset: float = 0.0, h_out=None, y_out=None, want_h=True, stream=None):
+    """x, residual (or None) fp16 CUDA [M, K], gamma fp16 [K] -> (h, y): h = x + residual, y = rmsnorm(h) * (gamma_offset + gamma).
+    h_out / y_out may be given (h_out may be x or residual: in place); want_h=False skips the h output (h is then None)."""
+    import torch
+    def ok(t, shape):
+        return t.dtype == torch.float16 and t.is_cuda and t.is_contiguous() and tuple(t.shape) == shape and t.device == x.device
+    if x.dim() != 2 or not ok(x, tuple(x.shape)) or x.shape[1] % 8 or x.shape[1] < 8:
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_residual_rmsnorm (x must be contiguous fp16 CUDA [M, K], K % 8 == 0)")
+    M, K = x.shape
+    if (residual is not None and not ok(residual, (M, K))) or not ok(gamma, (K,)):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_residual_rmsnorm (residual [M, K] / gamma [K] fp16 on x's device)")
+    if y_out is None:
+        y_out = torch.empty_like(x)
+    if h_out is None and want_h:
+        h_out = torch.empty_like(x)
+    if not ok(y_out, (M, K)) or (h_out is not None and not ok(h_out, (M, K))):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_residual_rmsnorm (bad output tensor)")
+    _check(lib.qlinear_residual_rmsnorm(ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(residual.data_ptr() if residual is not None else None),
+                                        ctypes.c_void_p(gamma.data_ptr()), float(eps), float(gamma_offset),
+                                        ctypes.c_void_p(h_out.data_ptr() if h_out is not None else None), ctypes.c_void_p(y_out.data_ptr()),
+                                        M, K, x.device.index or 0, _stream_ptr(stream)), "qlinear_residual_rmsnorm")
+    return h_out, y_out
 
 
 class QLinear:

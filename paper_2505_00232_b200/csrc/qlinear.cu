@@ -31,6 +31,7 @@ __device__ unsigned int* g_status_host;
 #include "gemm.cuh"
 #include "gemm_pair.cuh"
 #include "gemm_pair_ta.cuh"
+#include "norm.cuh"
 
 using namespace ql;
 
@@ -741,6 +742,36 @@ extern "C" ql_status qlinear_embed(qlinear_t h, const int32_t* ids, int32_t n, v
     if (L.bits == 8) embed_kernel<8, false><<<n, 128, 0, st>>>(prm);
     else if (L.grouped) embed_kernel<4, true><<<n, 128, 0, st>>>(prm);
     else embed_kernel<4, false><<<n, 128, 0, st>>>(prm);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_residual_rmsnorm(const void* x, const void* residual, const void* gamma, float eps, float gamma_offset,
+                                              void* h_out, void* y_out, int32_t M, int32_t K, int32_t device, void* stream)
+{
+    if (!x || !gamma || !y_out || M < 0 || K < 8 || (K % 8) || device < 0) return QL_ERR_INVALID_ARG;
+    if (!(eps >= 0.f) || y_out == h_out) return QL_ERR_INVALID_ARG;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(residual) | reinterpret_cast<uintptr_t>(gamma) |
+                          reinterpret_cast<uintptr_t>(h_out) | reinterpret_cast<uintptr_t>(y_out);
+    if (all & 15) return QL_ERR_INVALID_ARG;
+    if (M == 0) return QL_OK;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) { cudaGetLastError(); return QL_ERR_INVALID_ARG; }
+    DeviceGuard guard(device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    NormParams prm{};
+    prm.x = static_cast<const __half*>(x);
+    prm.r = static_cast<const __half*>(residual);
+    prm.g = static_cast<const __half*>(gamma);
+    prm.h_out = static_cast<__half*>(h_out);
+    prm.y_out = static_cast<__half*>(y_out);
+    prm.eps = eps; prm.offset = gamma_offset; prm.M = M; prm.K = K;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int vpt = (K / 8 + kNormThreads - 1) / kNormThreads;           // 8-value vectors per thread
+    if (vpt <= 1) residual_rmsnorm_kernel<1><<<M, kNormThreads, 0, st>>>(prm);
+    else if (vpt <= 2) residual_rmsnorm_kernel<2><<<M, kNormThreads, 0, st>>>(prm);
+    else if (vpt <= 4) residual_rmsnorm_kernel<4><<<M, kNormThreads, 0, st>>>(prm);
+    else if (vpt <= 8) residual_rmsnorm_kernel<8><<<M, kNormThreads, 0, st>>>(prm);
+    else residual_rmsnorm_kernel<0><<<M, kNormThreads, 0, st>>>(prm);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
