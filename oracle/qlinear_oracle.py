@@ -24,7 +24,7 @@ Parity pins: tests/test_oracle_pins.py (worked examples stored under
 tests/golden/, brute force over all byte values, one-hot / zero / closed-form
 cases, power-of-two and negation invariants, a double-rounding trap) and
 tests/test_oracle_pins_next.py for the three extensions further down (fused
-gating and residual + RMS normalisation, Section 3.6; int8 activation
+gating, residual + RMS normalisation and rotary embedding + QKV layout, Section 3.6; int8 activation
 quantisation, Section 3.7; the KV cache as weights, Section 3.8).  No function
 here is unpinned.
 """
@@ -284,6 +284,52 @@ def residual_rmsnorm_bound(h64, y64, K: int):
     bh = 2.0 ** -11 * np.abs(h64) + 2.0 ** -25
     by = (2.0 ** -11 + (K / 128.0 + 7 + 5) * 2.0 ** -24) * np.abs(y64) + 2.0 ** -25
     return bh, by
+
+
+# ----------------------------------------------------------------------------- rotary embedding + QKV layout (paper Section 3.6)
+# The paper's hand-written attention-block kernel "combine[s] rotary embedding with the layout transformations of query
+# (Q), key (K), and value (V) projections", the query going from (B, 1, S, h_q * d_h) to (B * h_kv, S * h_q / h_kv, d_h).
+# What the paper leaves open, and the readings taken (recorded in the design notes):
+#   * rotary convention: the rotate-half form of the paper's models (Llama, Gemma): element i < d_h / 2 pairs with
+#     element i + d_h / 2;  out_i = x_i * cos - x_{i+d/2} * sin,  out_{i+d/2} = x_{i+d/2} * cos + x_i * sin
+#   * the angles come as tables cos[p, i], sin[p, i] (fp32, one row per position p, i < d_h / 2) and a position per token,
+#     so that any frequency schedule can be used and no trigonometry is left to the kernel
+#   * order inside the merged query dimension: the source is (B, S, h_kv, g, d_h) with g = h_q / h_kv; the kernel swaps
+#     the S and h_kv axes, so row s * g + j of KV head hk holds query head hk * g + j of token s
+#   * K (rotated) and V (not rotated) go to (B * h_kv, S, d_h): one contiguous [S, d_h] block per KV head, the rows
+#     the KV cache of Section 3.8 takes in.
+def rope_qkv(q, k, v, pos, cos, sin, B: int, S: int, h_q: int, h_kv: int, d_h: int):
+    """q fp16 [B*S, h_q*d_h], k, v fp16 [B*S, h_kv*d_h], pos int [B*S], cos / sin fp32 [n_pos, d_h/2]
+    -> (q_out64 [B*h_kv, S*g, d_h], k_out64 [B*h_kv, S, d_h], v_out64 [B*h_kv, S, d_h], amp_q, amp_k) in fp64;
+    amp = |x_i| + |x_{i+d/2}| per output element (the tolerance denominator of the rotation)."""
+    g, half = h_q // h_kv, d_h // 2
+    assert h_q == g * h_kv and d_h == 2 * half
+    c = np.asarray(cos, dtype=np.float32).astype(np.float64)[np.asarray(pos)]           # [B*S, half]
+    s_ = np.asarray(sin, dtype=np.float32).astype(np.float64)[np.asarray(pos)]
+
+    def rotate(t, heads):
+        t = np.asarray(t, dtype=np.float16).astype(np.float64).reshape(B * S, heads, d_h)
+        lo, hi = t[:, :, :half], t[:, :, half:]
+        out = np.concatenate([lo * c[:, None, :] - hi * s_[:, None, :], hi * c[:, None, :] + lo * s_[:, None, :]], axis=2)
+        amp = np.concatenate([np.abs(lo) + np.abs(hi)] * 2, axis=2)
+        return out, amp
+
+    def to_heads(t, heads):                                              # [B*S, heads, d_h] -> [B, h_kv, S, heads / h_kv, d_h]
+        return t.reshape(B, S, h_kv, heads // h_kv, d_h).transpose(0, 2, 1, 3, 4)
+
+    rq, aq = rotate(q, h_q)
+    rk, ak = rotate(k, h_kv)
+    vv = np.asarray(v, dtype=np.float16).astype(np.float64).reshape(B * S, h_kv, d_h)
+    q_out = to_heads(rq, h_q).reshape(B * h_kv, S * g, d_h)
+    k_out = to_heads(rk, h_kv).reshape(B * h_kv, S, d_h)
+    v_out = to_heads(vv, h_kv).reshape(B * h_kv, S, d_h)
+    return q_out, k_out, v_out, to_heads(aq, h_q).reshape(B * h_kv, S * g, d_h), to_heads(ak, h_kv).reshape(B * h_kv, S, d_h)
+
+
+def rope_bound(y64, amp):
+    """|dy| allowed for an fp32 implementation: the fp16 rounding of the result (2^-11 relative, 2^-25 among the
+    subnormals) plus two products and one sum in fp32 (half an ulp of 2^-24 each, on terms no larger than amp)."""
+    return 2.0 ** -11 * np.abs(y64) + 3 * 2.0 ** -24 * amp + 2.0 ** -25
 
 
 # ----------------------------------------------------------------------------- C oracle

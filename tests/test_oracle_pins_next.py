@@ -310,3 +310,77 @@ def test_rmsnorm_bound_holds_for_an_fp32_emulation():
     h2, _, y2, _ = O.residual_rmsnorm(x[:, :K2], r[:, :K2], g[:K2], eps, 0.0)
     _, by2 = O.residual_rmsnorm_bound(h2, y2, K2)
     assert (np.abs(y2 * np.sqrt(K2 / (K2 - 1.0)) - y2) > by2).any()
+
+
+# ----------------------------------------------------------------------------- rotary embedding + QKV layout
+def test_example_J_rope_qkv(golden):
+    e = golden["J_rope_qkv"]
+    qo, ko, vo, _, _ = O.rope_qkv(np.array(e["q"], np.float16), np.array(e["k"], np.float16), np.array(e["v"], np.float16),
+                                  np.array(e["pos"]), np.array(e["cos"], np.float32), np.array(e["sin"], np.float32),
+                                  e["B"], e["S"], e["h_q"], e["h_kv"], e["d_h"])
+    assert (qo == np.array(e["q_out"])).all() and (ko == np.array(e["k_out"])).all() and (vo == np.array(e["v_out"])).all()
+
+
+def _rope_case(seed, B, S, h_q, h_kv, d_h, n_pos=64):
+    rng = np.random.default_rng(seed)
+    q = rng.standard_normal((B * S, h_q * d_h)).astype(np.float16)
+    k = rng.standard_normal((B * S, h_kv * d_h)).astype(np.float16)
+    v = rng.standard_normal((B * S, h_kv * d_h)).astype(np.float16)
+    pos = rng.integers(0, n_pos, size=B * S)
+    inv = 10000.0 ** (-np.arange(d_h // 2) * 2.0 / d_h)
+    ang = np.arange(n_pos)[:, None] * inv[None, :]
+    return q, k, v, pos, np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+
+
+def test_rope_layout_is_the_stated_index_map_and_v_is_only_moved():
+    B, S, h_q, h_kv, d_h = 2, 3, 6, 2, 4
+    g = h_q // h_kv
+    q, k, v, pos, cos, sin = _rope_case(1, B, S, h_q, h_kv, d_h)
+    one, zero = np.ones_like(cos), np.zeros_like(sin)                    # angle 0 everywhere: the pure layout transform
+    qo, ko, vo, _, _ = O.rope_qkv(q, k, v, pos, one, zero, B, S, h_q, h_kv, d_h)
+    for b in range(B):
+        for s in range(S):
+            for hk in range(h_kv):
+                assert (ko[b * h_kv + hk, s] == k[b * S + s, hk * d_h:(hk + 1) * d_h]).all()
+                assert (vo[b * h_kv + hk, s] == v[b * S + s, hk * d_h:(hk + 1) * d_h]).all()
+                for j in range(g):
+                    hq = hk * g + j
+                    assert (qo[b * h_kv + hk, s * g + j] == q[b * S + s, hq * d_h:(hq + 1) * d_h]).all()
+    _, _, vo2, _, _ = O.rope_qkv(q, k, v, pos, cos, sin, B, S, h_q, h_kv, d_h)
+    assert (vo2 == vo).all()                                             # V is never rotated
+
+
+def test_rope_is_the_complex_product_and_plain_loops():
+    B, S, h_q, h_kv, d_h = 1, 5, 4, 2, 8
+    half = d_h // 2
+    q, k, v, pos, cos, sin = _rope_case(2, B, S, h_q, h_kv, d_h)
+    qo, ko, _, aq, _ = O.rope_qkv(q, k, v, pos, cos, sin, B, S, h_q, h_kv, d_h)
+    g = h_q // h_kv
+    for s in range(S):
+        c, sn = cos[pos[s]].astype(np.float64), sin[pos[s]].astype(np.float64)
+        for hq in range(h_q):
+            x = q[s, hq * d_h:(hq + 1) * d_h].astype(np.float64)
+            z = (x[:half] + 1j * x[half:]) * (c + 1j * sn)               # the library's complex multiplication
+            row = qo[hq // g, s * g + hq % g]
+            np.testing.assert_allclose(row[:half], z.real, rtol=1e-15, atol=1e-300)
+            np.testing.assert_allclose(row[half:], z.imag, rtol=1e-15, atol=1e-300)
+            for i in range(half):                                        # and written out element by element
+                assert row[i] == x[i] * c[i] - x[i + half] * sn[i]
+                assert row[i + half] == x[i + half] * c[i] + x[i] * sn[i]
+                assert aq[hq // g, s * g + hq % g, i] == abs(x[i]) + abs(x[i + half])
+
+
+def test_rope_invariants():
+    B, S, h_q, h_kv, d_h = 1, 4, 2, 2, 16
+    half = d_h // 2
+    q, k, v, pos, cos, sin = _rope_case(3, B, S, h_q, h_kv, d_h)
+    qo, ko, _, _, _ = O.rope_qkv(q, k, v, pos, cos, sin, B, S, h_q, h_kv, d_h)
+    # a rotation keeps the length of every (i, i + d/2) pair (up to the rounding of the fp32 tables)
+    x = k.astype(np.float64).reshape(S, h_kv, d_h).transpose(1, 0, 2)
+    np.testing.assert_allclose(ko[:, :, :half] ** 2 + ko[:, :, half:] ** 2, x[:, :, :half] ** 2 + x[:, :, half:] ** 2, rtol=1e-6)
+    # the score of a query and a key depends on the DIFFERENCE of their positions only: shift all positions by 7
+    qo2, ko2, _, _, _ = O.rope_qkv(q, k, v, pos + 7, *_rope_case(3, B, S, h_q, h_kv, d_h, 80)[4:], B, S, h_q, h_kv, d_h)
+    np.testing.assert_allclose(np.einsum("hsd,htd->hst", qo2, ko2), np.einsum("hsd,htd->hst", qo, ko), rtol=0, atol=2e-5)
+    # the opposite sign of the sine table undoes the rotation
+    back = O.rope_qkv(np.zeros_like(q), ko.transpose(1, 0, 2).reshape(S, h_kv * d_h).astype(np.float16), v, pos, cos, -sin, B, S, h_q, h_kv, d_h)[1]
+    np.testing.assert_allclose(back.transpose(1, 0, 2).reshape(S, h_kv * d_h), k.astype(np.float64), rtol=0, atol=4e-3)
