@@ -633,6 +633,7 @@ def main():
                 line["configs"] += prefill_configs(torch, device, peaks, sidx, line)
                 line["fused_gating"] = gated_record(torch, device, peaks, sidx, ls)
                 line["residual_rmsnorm"] = norm_record(torch, device, peaks, sidx)
+                line["rope_qkv"] = rope_record(torch, device, peaks, sidx)
                 line["int8_activations"] = a8_record(torch, device, peaks, sidx)
         # ---- CPU oracle beside it (bounded sample)
         if not args.no_cpu_baseline:
@@ -694,6 +695,29 @@ def norm_record(torch, device, peaks, sidx):
         us = ms * 1e3 / (repeats * sets)
         gbs = 4 * M * K * 2 / 1e3 / us
         out[stage] = {"M": M, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
+    return out
+
+
+def rope_record(torch, device, peaks, sidx):
+    """Rotary embedding + Q/K/V layout transformation (paper Section 3.6) at the Llama3.1-8B head shape (32 / 8 heads of
+    128): prefill (S = 2048; 10 rotated buffer sets = 503 MB, past L2) and one decode token."""
+    import paper_2505_00232_b200 as P
+    h_q, h_kv, d_h, n_pos = 32, 8, 128, 4096
+    rng = np.random.default_rng(4)
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * (500000.0 ** (-np.arange(d_h // 2) * 2.0 / d_h))[None, :]
+    cos, sin = (torch.from_numpy(f(ang).astype(np.float32)).to(device) for f in (np.cos, np.sin))
+    out = {"h_q": h_q, "h_kv": h_kv, "d_h": d_h, "bytes_per_token": 2 * 2 * (h_q + 2 * h_kv) * d_h}
+    for stage, S, sets in (("prefill", 2048, 10), ("decode", 1, 64)):
+        mk = lambda heads: [torch.from_numpy(rng.standard_normal((S, heads * d_h)).astype(np.float16)).to(device) for _ in range(sets)]
+        qs, ks, vs = mk(h_q), mk(h_kv), mk(h_kv)
+        pos = torch.arange(S, dtype=torch.int32, device=device)
+        graph = capture_graph(torch, lambda i: P.qlinear_rope_qkv(qs[i], ks[i], vs[i], pos, cos, sin, 1, S, h_q, h_kv, d_h), sets)
+        for _ in range(3):
+            graph.replay()
+        ms, repeats, clocks = timed_region(torch, graph.replay, sets, sidx, 0.25)
+        us = ms * 1e3 / (repeats * sets)
+        gbs = out["bytes_per_token"] * S / 1e3 / us
+        out[stage] = {"S": S, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
     return out
 
 

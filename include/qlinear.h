@@ -237,6 +237,24 @@ ql_status qlinear_embed(qlinear_t h, const int32_t* ids_dev, int32_t n, void* y_
  * residual_dev (in place), y_out_dev may be x_dev; h_out_dev and y_out_dev must differ.  No handle, no library-owned
  * memory; asynchronous on cuda_stream.  Returns QL_ERR_INVALID_ARG for null / misaligned pointers or a bad shape,
  * QL_ERR_CUDA if the launch fails. */
+/* Rotary embedding combined with the layout transformation of the Q, K and V projections (paper Section 3.6: the
+ * hand-written kernel of the attention block; query from (B, 1, S, h_q * d_h) to (B * h_kv, S * h_q / h_kv, d_h)).
+ * Inputs (what the q / k / v projections wrote, token t = b * S + s): q_dev fp16 [B*S, h_q*d_h], k_dev and v_dev fp16
+ * [B*S, h_kv*d_h]; pos_dev int32 [B*S], the position of every token; cos_dev / sin_dev fp32 [n_pos, d_h/2], the angle
+ * tables (row = position), so that any frequency schedule can be used.  The paper fixes neither the rotary convention
+ * nor the order inside the merged query dimension; the readings taken: rotate-half pairs (element i < d_h/2 with
+ * element i + d_h/2:  out_i = x_i cos - x_{i+d/2} sin,  out_{i+d/2} = x_{i+d/2} cos + x_i sin), and, with g = h_q / h_kv,
+ *     q_out[b*h_kv + hk, s*g + j, :] = rot(q[t, (hk*g + j)*d_h ...]),   k_out[b*h_kv + hk, s, :] = rot(k[t, hk*d_h ...]),
+ *     v_out[b*h_kv + hk, s, :] = v[t, hk*d_h ...]   (not rotated),
+ * i.e. one contiguous [rows, d_h] block per KV head: the rows qlinear_kv_append and qlinear_kv_scores take.
+ * q_out_dev fp16 [B*h_kv, S*g, d_h], k_out_dev and v_out_dev fp16 [B*h_kv, S, d_h]; all pointers device memory of
+ * `device`, 16-byte aligned (pos 4); outputs must not be the inputs.  h_q a multiple of h_kv, d_h a multiple of 16;
+ * positions must lie in [0, n_pos) (the kernel clamps them rather than read outside the tables).  No handle, no
+ * library-owned memory; asynchronous on cuda_stream.  QL_ERR_INVALID_ARG for null / misaligned pointers or bad shapes. */
+ql_status qlinear_rope_qkv(const void* q_dev, const void* k_dev, const void* v_dev, const int32_t* pos_dev, const float* cos_dev,
+                           const float* sin_dev, int32_t n_pos, void* q_out_dev, void* k_out_dev, void* v_out_dev, int32_t B, int32_t S,
+                           int32_t h_q, int32_t h_kv, int32_t d_h, int32_t device, void* cuda_stream);
+
 ql_status qlinear_residual_rmsnorm(const void* x_dev, const void* residual_dev, const void* gamma_dev, float eps, float gamma_offset,
                                    void* h_out_dev, void* y_out_dev, int32_t M, int32_t K, int32_t device, void* cuda_stream);
 

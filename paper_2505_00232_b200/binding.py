@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -78,6 +78,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_embed.restype = ctypes.c_int
     lib.qlinear_residual_rmsnorm.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp, i32, i32, ctypes.c_int, vp]
     lib.qlinear_residual_rmsnorm.restype = ctypes.c_int
+    lib.qlinear_rope_qkv.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, ctypes.c_int, vp]
+    lib.qlinear_rope_qkv.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
     lib.qlinear_debug_expire_wait.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -264,6 +266,27 @@ def qlinear_residual_rmsnorm(x, residual, gamma, eps: float, gamma_offset: float
                                         ctypes.c_void_p(h_out.data_ptr() if h_out is not None else None), ctypes.c_void_p(y_out.data_ptr()),
                                         M, K, x.device.index or 0, _stream_ptr(stream)), "qlinear_residual_rmsnorm")
     return h_out, y_out
+
+
+def qlinear_rope_qkv(q, k, v, pos, cos, sin, B: int, S: int, h_q: int, h_kv: int, d_h: int, stream=None):
+    """q fp16 CUDA [B*S, h_q*d_h], k, v [B*S, h_kv*d_h], pos int32 [B*S], cos / sin fp32 [n_pos, d_h/2]
+    -> (q_out [B*h_kv, S*h_q/h_kv, d_h], k_out [B*h_kv, S, d_h], v_out [B*h_kv, S, d_h]): rotary embedding + layout change."""
+    import torch
+    T = B * S
+    def ok(t, dtype, shape):
+        return t.dtype == dtype and t.is_cuda and t.is_contiguous() and tuple(t.shape) == shape and t.device == q.device
+    if h_kv < 1 or h_q % h_kv or d_h % 16 or not ok(q, torch.float16, (T, h_q * d_h)) or not ok(k, torch.float16, (T, h_kv * d_h)) \
+            or not ok(v, torch.float16, (T, h_kv * d_h)) or not ok(pos, torch.int32, (T,)) or cos.dim() != 2 \
+            or not ok(cos, torch.float32, (cos.shape[0], d_h // 2)) or not ok(sin, torch.float32, tuple(cos.shape)):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_rope_qkv (shapes / dtypes: see the header)")
+    g = h_q // h_kv
+    q_out = torch.empty((B * h_kv, S * g, d_h), dtype=torch.float16, device=q.device)
+    k_out = torch.empty((B * h_kv, S, d_h), dtype=torch.float16, device=q.device)
+    v_out = torch.empty((B * h_kv, S, d_h), dtype=torch.float16, device=q.device)
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    _check(lib.qlinear_rope_qkv(p(q), p(k), p(v), p(pos), p(cos), p(sin), cos.shape[0], p(q_out), p(k_out), p(v_out), B, S, h_q, h_kv, d_h,
+                                q.device.index or 0, _stream_ptr(stream)), "qlinear_rope_qkv")
+    return q_out, k_out, v_out
 
 
 class QLinear:

@@ -32,6 +32,7 @@ __device__ unsigned int* g_status_host;
 #include "gemm_pair.cuh"
 #include "gemm_pair_ta.cuh"
 #include "norm.cuh"
+#include "rope.cuh"
 
 using namespace ql;
 
@@ -772,6 +773,31 @@ extern "C" ql_status qlinear_residual_rmsnorm(const void* x, const void* residua
     else if (vpt <= 4) residual_rmsnorm_kernel<4><<<M, kNormThreads, 0, st>>>(prm);
     else if (vpt <= 8) residual_rmsnorm_kernel<8><<<M, kNormThreads, 0, st>>>(prm);
     else residual_rmsnorm_kernel<0><<<M, kNormThreads, 0, st>>>(prm);
+    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
+extern "C" ql_status qlinear_rope_qkv(const void* q, const void* k, const void* v, const int32_t* pos, const float* cos_t, const float* sin_t,
+                                      int32_t n_pos, void* q_out, void* k_out, void* v_out, int32_t B, int32_t S, int32_t h_q, int32_t h_kv,
+                                      int32_t d_h, int32_t device, void* stream)
+{
+    if (!q || !k || !v || !pos || !cos_t || !sin_t || !q_out || !k_out || !v_out) return QL_ERR_INVALID_ARG;
+    if (B < 0 || S < 0 || h_q < 1 || h_kv < 1 || (h_q % h_kv) || d_h < 16 || (d_h % 16) || n_pos < 1 || device < 0) return QL_ERR_INVALID_ARG;
+    if ((int64_t)B * S > INT32_MAX || (int64_t)B * S * h_q * d_h > ((int64_t)1 << 40)) return QL_ERR_INVALID_ARG;
+    const uintptr_t all = reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k) | reinterpret_cast<uintptr_t>(v) | reinterpret_cast<uintptr_t>(cos_t) |
+                          reinterpret_cast<uintptr_t>(sin_t) | reinterpret_cast<uintptr_t>(q_out) | reinterpret_cast<uintptr_t>(k_out) | reinterpret_cast<uintptr_t>(v_out);
+    if ((all & 15) || (reinterpret_cast<uintptr_t>(pos) & 3)) return QL_ERR_INVALID_ARG;
+    if (q_out == q || k_out == k || v_out == v) return QL_ERR_INVALID_ARG;   // the layout changes: not in place
+    if ((int64_t)B * S == 0) return QL_OK;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device >= n_dev) { cudaGetLastError(); return QL_ERR_INVALID_ARG; }
+    DeviceGuard guard(device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    RopeParams prm{};
+    prm.q = static_cast<const __half*>(q); prm.k = static_cast<const __half*>(k); prm.v = static_cast<const __half*>(v);
+    prm.pos = pos; prm.cos_t = cos_t; prm.sin_t = sin_t;
+    prm.q_out = static_cast<__half*>(q_out); prm.k_out = static_cast<__half*>(k_out); prm.v_out = static_cast<__half*>(v_out);
+    prm.B = B; prm.S = S; prm.h_q = h_q; prm.h_kv = h_kv; prm.d_h = d_h; prm.n_pos = n_pos;
+    rope_qkv_kernel<<<B * S, kRopeThreads, 0, static_cast<cudaStream_t>(stream)>>>(prm);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
