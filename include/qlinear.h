@@ -135,6 +135,13 @@ ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
 
+/* Layers with DIFFERENT inputs in one launch: ys[i] = xs[i] . W_i^T for i < n (1 <= n <= 4), all with the same M.  The
+ * case in mind is the attention products over the KV cache held as weights (paper Section 3.8): every KV head has its
+ * own cache handle and its own query rows, and a launch per head and product is launch-bound.  Same requirements on the
+ * handles as qlinear_forward_group (one device, equal K, bits and group).  For M <= 8 and K a whole number of chunks the
+ * call is one decode launch; otherwise it is n calls of qlinear_forward, in order.  Pointers as for qlinear_forward. */
+ql_status qlinear_forward_batch(const qlinear_t* handles, int32_t n, const void* const* xs_dev, void* const* ys_dev, int32_t M, void* cuda_stream);
+
 /* Activation of the gate branch in qlinear_forward_gated. */
 typedef enum { QL_ACT_IDENTITY = 0, QL_ACT_SILU = 1, QL_ACT_GELU_TANH = 2 } ql_act;
 

@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_batch", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -62,6 +62,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_debug_unpack_device.restype = ctypes.c_int
     lib.qlinear_forward_group.argtypes = [ctypes.POINTER(vp), ctypes.c_int32, vp, ctypes.POINTER(vp), ctypes.c_int32, vp]
     lib.qlinear_forward_group.restype = ctypes.c_int
+    lib.qlinear_forward_batch.argtypes = [ctypes.POINTER(vp), ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int32, vp]
+    lib.qlinear_forward_batch.restype = ctypes.c_int
     lib.qlinear_forward_gated.argtypes = [vp, vp, vp, vp, i32, i32, vp]
     lib.qlinear_forward_gated.restype = ctypes.c_int
     lib.qlinear_forward_a8.argtypes = [vp, vp, vp, i32, vp]
@@ -191,6 +193,38 @@ def qlinear_forward_group_raw(lins, x_ptr: int, y_ptrs, M: int, stream=None) -> 
     hs = (ctypes.c_void_p * n)(*[l._h for l in lins])
     ys = (ctypes.c_void_p * n)(*[ctypes.c_void_p(int(p)) for p in y_ptrs])
     _check(lib.qlinear_forward_group(hs, n, ctypes.c_void_p(x_ptr), ys, M, _stream_ptr(stream)), "qlinear_forward_group")
+
+
+def qlinear_forward_batch_raw(lins, x_ptrs, y_ptrs, M: int, stream=None) -> None:
+    """qlinear_forward_batch on raw device pointers: layer i applied to its own input x_ptrs[i]."""
+    n = len(lins)
+    hs = (ctypes.c_void_p * n)(*[l._h for l in lins])
+    xs = (ctypes.c_void_p * n)(*[ctypes.c_void_p(int(p)) for p in x_ptrs])
+    ys = (ctypes.c_void_p * n)(*[ctypes.c_void_p(int(p)) for p in y_ptrs])
+    _check(lib.qlinear_forward_batch(hs, n, xs, ys, M, _stream_ptr(stream)), "qlinear_forward_batch")
+
+
+def qlinear_forward_batch(lins, xs, outs=None, stream=None):
+    """xs: one fp16 CUDA tensor [M, K] per layer -> list of fp16 [M, N_i] (one launch for M <= 8, up to 4 layers)."""
+    import torch
+    K, M = lins[0].desc.K, xs[0].shape[0]
+    if len(xs) != len(lins):
+        raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_batch (one input per layer)")
+    for x in xs:
+        if x.dim() != 2 or tuple(x.shape) != (M, K) or x.dtype != torch.float16 or not x.is_cuda or not x.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_batch (every x must be contiguous fp16 CUDA [M, K])")
+    if outs is None:
+        outs = [torch.empty((M, l.desc.N), dtype=torch.float16, device=xs[0].device) for l in lins]
+    for l, o in zip(lins, outs):
+        if o.shape != (M, l.desc.N) or o.dtype != torch.float16 or not o.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_forward_batch (bad out tensor)")
+    qlinear_forward_batch_raw(lins, [x.data_ptr() for x in xs], [o.data_ptr() for o in outs], M, stream)
+    return outs
+
+
+def kv_scores_batch(caches, q_rows, stream=None):
+    """The score product of up to 4 KV heads in one launch: caches[i].scores(q_rows[i]) for every i (paper Section 3.8)."""
+    return qlinear_forward_batch([c.k for c in caches], q_rows, stream=stream)
 
 
 def qlinear_forward_group(lins, x, outs=None, stream=None):

@@ -40,6 +40,9 @@ struct GemvParams {
     int32_t rb_end[kGemvMaxGroup];
     int32_t n_layers;
     const __half* x;                     // [M, K]
+    // Batched form (layers with DIFFERENT inputs in one launch, e.g. the score products of several KV heads): the input
+    // of layer i; the plain and grouped forms set every entry to x.  Only the direct form (XDIRECT) reads it per layer.
+    const __half* xl[kGemvMaxGroup];
     int32_t M, K;
     int32_t n_rb;                        // row-blocks holding at least one real row, all layers
     int32_t n_kc;                        // chunks along K
@@ -145,7 +148,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     float total[4] = {0.f, 0.f, 0.f, 0.f};
     // Lanes whose token column does not exist (g >= M) read the last real token: MMA columns are
     // independent and those columns are never stored.
-    const __half* xpass = XDIRECT ? p.x + (int64_t)min(g, p.M - 1) * p.K + 8 * c + kc0 * CHUNK_K
+    const __half* xpass = XDIRECT ? p.xl[layer] + (int64_t)min(g, p.M - 1) * p.K + 8 * c + kc0 * CHUNK_K
                                   : xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
     // Direct form: the host chooses it only when K is a whole number of chunks, so every chunk in
     // [kc0, kc1) lies inside the token's row and the loads need no bounds check.

@@ -245,7 +245,10 @@ cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPla
 // One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
 // call (integer arithmetic only); nothing is written to a handle.
 // act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
-ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1)
+// xs != nullptr: the batched form, layer i reads xs[i] (x is then ignored); needs the kernel form that reads x straight
+// from global memory.
+ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1,
+                       const void* const* xs = nullptr)
 {
     const qlinear_s* h = hs[0];
     const Layout& L = h->L;
@@ -254,7 +257,7 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     const bool gated = act >= 0;
     if (gated) n_rb = 2 * hs[0]->n_rb;
     const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
-    if (gated && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
+    if ((gated || xs) && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
     cudaError_t e;
     if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
     GemvParams prm{};
@@ -270,7 +273,8 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     }
     prm.n_layers = n;
     prm.act = gated ? act : 0;
-    prm.x = static_cast<const __half*>(x);
+    prm.x = static_cast<const __half*>(xs ? xs[0] : x);
+    for (int i = 0; i < kGemvMaxGroup; ++i) prm.xl[i] = static_cast<const __half*>(xs ? xs[i < n ? i : 0] : x);
     prm.M = M; prm.K = L.K;
     prm.n_rb = n_rb;
     prm.n_kc = L.n_kc;
@@ -554,6 +558,29 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
     }
     for (int i = 0; i < n; ++i) {
         ql_status s = qlinear_forward(hs[i], x, ys[i], M, stream);
+        if (s != QL_OK) return s;
+    }
+    return QL_OK;
+}
+
+extern "C" ql_status qlinear_forward_batch(const qlinear_t* hs, int32_t n, const void* const* xs, void* const* ys, int32_t M, void* stream)
+{
+    if (!hs || !xs || !ys || n < 1 || n > kGemvMaxGroup || M < 1) return QL_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i) {
+        if (!hs[i] || !xs[i] || !ys[i] || ((reinterpret_cast<uintptr_t>(xs[i]) | reinterpret_cast<uintptr_t>(ys[i])) & 15)) return QL_ERR_INVALID_ARG;
+        const Layout &a = hs[0]->L, &b = hs[i]->L;
+        if (hs[i]->device != hs[0]->device || a.K != b.K || a.bits != b.bits || a.group != b.group) return QL_ERR_INVALID_ARG;
+        if ((int64_t)M * b.N > INT32_MAX || (int64_t)M * b.K > INT32_MAX) return QL_ERR_INVALID_ARG;
+    }
+    if (device_timed_out(hs[0])) return QL_ERR_DEVICE_TIMEOUT;
+    if (n > 1 && M <= hs[0]->gemv_max_m && !hs[0]->use_stream) {         // one decode launch for all of them
+        DeviceGuard guard(hs[0]->device);
+        if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+        const ql_status s = forward_gemv(const_cast<qlinear_s* const*>(hs), n, nullptr, ys, M, static_cast<cudaStream_t>(stream), -1, xs);
+        if (s != QL_ERR_UNSUPPORTED) return s;
+    }
+    for (int i = 0; i < n; ++i) {                                        // anything else: one call per layer
+        const ql_status s = qlinear_forward(hs[i], xs[i], ys[i], M, stream);
         if (s != QL_OK) return s;
     }
     return QL_OK;
