@@ -824,7 +824,11 @@ extern "C" ql_status qlinear_rope_qkv(const void* q, const void* k, const void* 
     prm.pos = pos; prm.cos_t = cos_t; prm.sin_t = sin_t;
     prm.q_out = static_cast<__half*>(q_out); prm.k_out = static_cast<__half*>(k_out); prm.v_out = static_cast<__half*>(v_out);
     prm.B = B; prm.S = S; prm.h_q = h_q; prm.h_kv = h_kv; prm.d_h = d_h; prm.n_pos = n_pos;
-    rope_qkv_kernel<<<B * S, kRopeThreads, 0, static_cast<cudaStream_t>(stream)>>>(prm);
+    // threads: the work items of a token (8-element vectors of half a head) spread evenly over the fewest passes
+    const int items = (h_q + h_kv) * (d_h / 16) + h_kv * (d_h / 8);
+    const int passes = (items + kRopeThreads - 1) / kRopeThreads;
+    const int threads = std::min(kRopeThreads, (((items + passes - 1) / passes) + 31) / 32 * 32);
+    rope_qkv_kernel<<<B * S, threads, 0, static_cast<cudaStream_t>(stream)>>>(prm);
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 

@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kRopeThreads) rope_qkv_kernel(const RopeParams
     const int rot_items = (p.h_q + p.h_kv) * vec_half;
     const int items = rot_items + p.h_kv * 2 * vec_half;
 
-    for (int it = threadIdx.x; it < items; it += kRopeThreads) {
+    for (int it = threadIdx.x; it < items; it += blockDim.x) {
         if (it < rot_items) {
             const int head = it / vec_half, i0 = (it - head * vec_half) << 3;       // q heads first, then k heads
             const bool is_q = head < p.h_q;
