@@ -59,6 +59,9 @@ __global__ void __launch_bounds__(kNormThreads) residual_rmsnorm_kernel(const No
     const int n_vec = p.K >> 3;
     constexpr int NV = VPT > 0 ? VPT : 1;
     float keep[NV][8];
+    // programmatic dependent launch: the next kernel may start its own set-up now; x and r may come from the previous one
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     auto load_h = [&](int v, float a[8]) {
         norm_load8(p.x + row + 8 * v, a);

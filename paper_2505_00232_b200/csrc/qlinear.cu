@@ -795,12 +795,15 @@ extern "C" ql_status qlinear_residual_rmsnorm(const void* x, const void* residua
     prm.eps = eps; prm.offset = gamma_offset; prm.M = M; prm.K = K;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int vpt = (K / 8 + kNormThreads - 1) / kNormThreads;           // 8-value vectors per thread
-    if (vpt <= 1) residual_rmsnorm_kernel<1><<<M, kNormThreads, 0, st>>>(prm);
-    else if (vpt <= 2) residual_rmsnorm_kernel<2><<<M, kNormThreads, 0, st>>>(prm);
-    else if (vpt <= 4) residual_rmsnorm_kernel<4><<<M, kNormThreads, 0, st>>>(prm);
-    else if (vpt <= 8) residual_rmsnorm_kernel<8><<<M, kNormThreads, 0, st>>>(prm);
-    else residual_rmsnorm_kernel<0><<<M, kNormThreads, 0, st>>>(prm);
-    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+    const bool pdl = config().pdl;
+    cudaError_t e;
+    if (vpt <= 1) e = launch(residual_rmsnorm_kernel<1>, prm, dim3(M), dim3(kNormThreads), 0, st, 1, pdl);
+    else if (vpt <= 2) e = launch(residual_rmsnorm_kernel<2>, prm, dim3(M), dim3(kNormThreads), 0, st, 1, pdl);
+    else if (vpt <= 4) e = launch(residual_rmsnorm_kernel<4>, prm, dim3(M), dim3(kNormThreads), 0, st, 1, pdl);
+    else if (vpt <= 8) e = launch(residual_rmsnorm_kernel<8>, prm, dim3(M), dim3(kNormThreads), 0, st, 1, pdl);
+    else e = launch(residual_rmsnorm_kernel<0>, prm, dim3(M), dim3(kNormThreads), 0, st, 1, pdl);
+    if (e != cudaSuccess) cudaGetLastError();
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
 extern "C" ql_status qlinear_rope_qkv(const void* q, const void* k, const void* v, const int32_t* pos, const float* cos_t, const float* sin_t,
@@ -828,8 +831,9 @@ extern "C" ql_status qlinear_rope_qkv(const void* q, const void* k, const void* 
     const int items = (h_q + h_kv) * (d_h / 16) + h_kv * (d_h / 8);
     const int passes = (items + kRopeThreads - 1) / kRopeThreads;
     const int threads = std::min(kRopeThreads, (((items + passes - 1) / passes) + 31) / 32 * 32);
-    rope_qkv_kernel<<<B * S, threads, 0, static_cast<cudaStream_t>(stream)>>>(prm);
-    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+    const cudaError_t e = launch(rope_qkv_kernel, prm, dim3(B * S), dim3(threads), 0, static_cast<cudaStream_t>(stream), 1, config().pdl);
+    if (e != cudaSuccess) cudaGetLastError();
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
 extern "C" ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_out, void* stream)

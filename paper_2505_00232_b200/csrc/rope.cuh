@@ -48,6 +48,8 @@ __device__ __forceinline__ uint4 rope_pack8(const float f[8])
 
 __global__ void __launch_bounds__(kRopeThreads) rope_qkv_kernel(const RopeParams p)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may set up; q, k, v may come from the previous one
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int t = blockIdx.x, b = t / p.S, s = t - b * p.S;
     const int g = p.h_q / p.h_kv, half = p.d_h >> 1, vec_half = half >> 3;
     const int pos = min(max(p.pos[t], 0), p.n_pos - 1);                  // (the caller keeps positions inside the tables)

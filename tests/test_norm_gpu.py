@@ -98,3 +98,40 @@ def test_bad_arguments(P, torch):
         P.qlinear_residual_rmsnorm(x, None, g, 1e-5, h_out=x, y_out=x)   # the two outputs must differ
     with pytest.raises(P.QLinearError):
         P.qlinear_residual_rmsnorm(x, None, g, -1.0)
+
+
+def test_chain_with_linear_layers_needs_no_synchronisation(P, torch):
+    """norm -> linear -> norm -> linear on one stream, decode and prefill sizes, buffers reused: every kernel releases its
+    successor early (programmatic dependent launch), so the unsynchronised chain must give the bits of the synchronised one."""
+    from workloads import configs as C
+    K = 2048
+    spec = C.LayerSpec("t", K, K, 4, 32, -8, 7)
+    lins = []
+    for i in range(2):
+        q, s = C.layer_weights(70 + i, spec)
+        lins.append(P.QLinear.from_weights(q, (s.astype(np.float32) / 8).astype(np.float16), 4, 32, device="cuda:0"))
+    g = torch.from_numpy(inputs(1, 1, K)[2]).cuda()
+    for M in (1, 4, 300):
+        x0 = torch.from_numpy(inputs(2 + M, M, K)[0]).cuda()
+        res = torch.zeros((M, K), dtype=torch.float16, device="cuda")
+        a = torch.empty_like(res)
+        b = torch.empty_like(res)
+
+        def chain(sync):
+            res.zero_()
+            cur = x0
+            for lin in lins:
+                P.qlinear_residual_rmsnorm(cur, res, g, 1e-5, 1.0, h_out=res, y_out=a)
+                if sync:
+                    torch.cuda.synchronize()
+                lin.forward_raw(a.data_ptr(), b.data_ptr(), M)
+                if sync:
+                    torch.cuda.synchronize()
+                cur = b
+            torch.cuda.synchronize()
+            return res.clone(), b.clone()
+
+        ref = chain(True)
+        for _ in range(4):
+            got = chain(False)
+            assert all(torch.equal(r.view(torch.int16), o.view(torch.int16)) for r, o in zip(ref, got))
