@@ -24,9 +24,14 @@
 //     on which the slot's 8 warps, the step's x tile and the peer CTA arrive, so that the issuing thread waits once
 //     per k-step.
 //
-// What bounds it (measured): not the tensor pipe (halving the MMA width changes nothing) but the instruction stream
+// What bounded it (measured): not the tensor pipe (halving the MMA width changed nothing) but the instruction stream
 // of the dequantise warps and of the polling threads around them, which is why every warp loops over its own steps
-// only and no thread polls in the main loop.
+// only and no thread polls in the main loop.  As it stands the tensor pipe is active 86-91 % of the cycles in which an
+// SM has work, at the clock the power limit leaves.
+//
+// Forms of the kernel (template flags): the plain product, whole tiles dealt out round-robin or, for launches with
+// few tiles, 2 or 4 K parts per tile that meet in the device scratch; GATED (y = act(gate) * up, Section 3.6); I8
+// (int8 activations, kind::i8 on the stored weight bytes, Section 3.7).
 //
 // Protocol between the two CTAs: own loads only; the leader issues; commits are multicast to both CTAs; the peer relays
 // "slot ready" (see the relay below).
