@@ -626,6 +626,8 @@ def main():
             # that follow heat the part and would lower the clocks of whatever runs after them)
             if not args.no_configs:
                 line["configs"] = decode_configs(torch, device, peaks, sidx, ls, line)
+                if {"q", "k", "v", "o", "gate", "up", "down"} <= {l.name for l in ls.workload.layers} and ls.M <= 8:
+                    line["decoder_block"] = block_record(torch, device, peaks, sidx, ls)
             # ---- second stage of the hot path on the SAME resident weights (copy 0), measured in the same run
             if not args.no_prefill:
                 line["prefill"] = prefill_sub(torch, device, peaks, args.prefill_steps, sidx, ls.blob0)
@@ -719,6 +721,48 @@ def rope_record(torch, device, peaks, sidx):
         gbs = out["bytes_per_token"] * S / 1e3 / us
         out[stage] = {"S": S, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
     return out
+
+
+def block_record(torch, device, peaks, sidx, ls_main):
+    """The linear hot path of ONE Llama3.1-8B transformer block at the headline's M with the operators of Section 3.6
+    around it, chained on one stream the way a decoder issues them (the attention core itself is not part of this
+    library and is left out: the o projection reads a buffer of the right shape):
+      residual + rmsnorm -> q/k/v (one grouped launch) -> rotary + QKV layout -> o -> residual + rmsnorm
+      -> gate/up with the gating fused -> down.
+    8 kernels, replayed as one CUDA graph over the rotated weight copies; value = weight bytes over time."""
+    import paper_2505_00232_b200 as P
+    w, M, copies = ls_main.workload, ls_main.M, ls_main.copies
+    idx = {l.name: i for i, l in enumerate(w.layers)}
+    D, h_q, h_kv, d_h = w.layers[idx["q"]].K, 32, 8, 128
+    rng = np.random.default_rng(11)
+    f16 = lambda *shape: torch.from_numpy(rng.standard_normal(shape).astype(np.float16)).to(device)
+    x, res, gam = f16(M, D), f16(M, D), f16(D)
+    a, attn = torch.empty_like(x), f16(M, h_q * d_h)
+    yq, yk, yv = (torch.empty((M, n), dtype=torch.float16, device=device) for n in (h_q * d_h, h_kv * d_h, h_kv * d_h))
+    x2 = torch.empty_like(x)
+    ff = torch.empty((M, w.layers[idx["gate"]].N), dtype=torch.float16, device=device)
+    pos = torch.arange(M, dtype=torch.int32, device=device)
+    ang = np.arange(64, dtype=np.float64)[:, None] * (500000.0 ** (-np.arange(d_h // 2) * 2.0 / d_h))[None, :]
+    cos, sin = (torch.from_numpy(f(ang).astype(np.float32)).to(device) for f in (np.cos, np.sin))
+
+    def block(cp):
+        L = ls_main.lin[cp]
+        P.qlinear_residual_rmsnorm(x, res, gam, 1e-5, 0.0, h_out=res, y_out=a)
+        P.qlinear_forward_group_raw([L[idx["q"]], L[idx["k"]], L[idx["v"]]], a.data_ptr(), [yq.data_ptr(), yk.data_ptr(), yv.data_ptr()], M)
+        P.qlinear_rope_qkv(yq, yk, yv, pos, cos, sin, 1, M, h_q, h_kv, d_h)
+        L[idx["o"]].forward_raw(attn.data_ptr(), x2.data_ptr(), M)
+        P.qlinear_residual_rmsnorm(x2, res, gam, 1e-5, 0.0, h_out=res, y_out=a)
+        P.qlinear_forward_gated_raw(L[idx["gate"]], L[idx["up"]], a.data_ptr(), ff.data_ptr(), M, "silu")
+        L[idx["down"]].forward_raw(ff.data_ptr(), x.data_ptr(), M)
+
+    graph = capture_graph(torch, lambda i: block(i % copies), copies)
+    for _ in range(3):
+        graph.replay()
+    ms, repeats, clocks = timed_region(torch, graph.replay, copies, sidx, 0.25)
+    us = ms * 1e3 / (repeats * copies)
+    gbs = ls_main.weight_bytes / 1e3 / us
+    return {"M": M, "kernels": 8, "us": us, "weight_gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"],
+            "note": "residual+rmsnorm, q/k/v grouped, rope+layout, o, residual+rmsnorm, gated gate/up, down; attention core not included"}
 
 
 def gated_record(torch, device, peaks, sidx, ls_main):
