@@ -66,6 +66,9 @@ struct GemmTaSmem {
     static constexpr int kXStages = (I8 && BITS == 8) ? 6 : 7;           // <= kASlots: the x producer reads "stage free" off the A-slot barrier
     static constexpr int kWBlocks = (I8 ? 2 : 1) * (BITS == 4 ? 1 : 2);  // packed blocks per k-step
     static constexpr int kWBytes = I8 ? kWBlocks * kWeightBlockBytes : (BITS == 4 ? 5120 : 8192);
+    // A ring length that is a multiple of the 3 dequantise turns keeps every stage with one turn, whose warps then see all
+    // of the stage's phases in order; the 16 KB stages of the int8 integer form leave room for 4 only, and its warps first
+    // wait for the stage's release (see the main loop of the dequantise warps).
     static constexpr int kWStages = I8 ? (BITS == 4 ? 6 : 4) : (BITS == 4 ? 9 : 6);
     static constexpr int kASlots = 8;                                    // tensor memory: 8 x 32 columns beside the accumulator
     static constexpr int kEarlySteps = kASlots - 2;                      // steps of the next tile dequantised before the epilogue is forced
@@ -578,6 +581,11 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                 if (!ok) break;
             }
             uint32_t r[16];
+            // A weight stage whose ring length is not a multiple of the 3 turns is served by a different turn every time
+            // round, so this warp has not seen the stage's previous phase: the load of step g - NW may still be in flight
+            // (bulk copies complete in any order), and a parity test alone would then take that phase for this one.  The
+            // producer issues the load of step g only after step g - NW's warps have released the stage: wait for that first.
+            if (NW % 3 != 0 && !mbar_wait(wempty_bar(s), wpar ^ 1, abort_flag, 0x480 + s)) { ok = false; break; }
             if (!mbar_wait(wfull_bar(s), wpar, abort_flag, 0x400 + s)) { ok = false; break; }
             if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED, I8>(wpk_addr(s), half, r);
             else {

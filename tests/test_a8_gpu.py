@@ -150,6 +150,26 @@ def test_a8_prefill_llama_shapes_full_size(P, torch, name, bits):
         assert_a8(y[:, r0:r0 + 2048], x, q[r0:r0 + 2048], s[r0:r0 + 2048], 0)
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+def test_a8_prefill_back_to_back_launches_keep_their_bits(P, torch, bits):
+    """Several thousand integer-form launches in a row from two handles, without host synchronisation in between: no
+    bounded wait expires and every sampled output has the bits of the first one.  (The weight ring of the int8 form is
+    not a multiple of the three dequantise turns long; a warp that takes a stage's previous phase for its own reads stale
+    bytes and leaves the ring one arrival short, which shows up only under particular load timings.)"""
+    N, K, M = 4096, 4096, 2048
+    q, s, x = rand_case(7500 + bits, M, N, K, bits, 0)
+    lins = [P.QLinear.from_weights(q, s, bits, 0, device="cuda:0") for _ in range(2)]
+    xd = torch.from_numpy(x).cuda()
+    y = torch.empty((M, N), dtype=torch.float16, device="cuda:0")
+    first = lins[0].forward_a8(xd).clone()
+    for rnd in range(6):
+        for i in range(500):
+            lins[i & 1].forward_a8_raw(xd.data_ptr(), y.data_ptr(), M)
+        assert torch.equal(y, first), f"round {rnd}"
+    torch.cuda.synchronize()
+    assert lins[0].device_status() == (0, 0)
+
+
 def test_a8_zero_input_and_guard_bands(P, torch):
     q, s, x = rand_case(7100, 3, 200, 352, 4, 32)
     lin = P.QLinear.from_weights(q, s, 4, 32, device="cuda:0")
