@@ -140,3 +140,28 @@ def test_dependent_launches_back_to_back(P, torch):
         for r, g in zip(ref, got):
             assert torch.equal(r.view(torch.int16), g.view(torch.int16))
     assert lins[0].device_status() == (0, 0)
+
+
+# (M, N, K, bits, group): whole tiles round-robin (two ring lengths), a K split of 4 and of 2 parts through the scratch,
+# a launch of at most 128 tokens
+STRESS = [(2048, 4096, 4096, 4, 32), (2048, 4096, 4096, 8, 0), (1024, 2304, 9216, 4, 32), (512, 4864, 2048, 8, 0), (64, 4096, 14336, 4, 0)]
+
+
+@pytest.mark.parametrize("M,N,K,bits,group", STRESS)
+def test_back_to_back_launches_keep_their_bits(P, torch, M, N, K, bits, group):
+    """A few thousand launches in a row from two handles without host synchronisation (the pipelines of consecutive
+    launches overlap, loads land in whatever order the memory system returns them): no bounded wait expires and every
+    sampled output has the bits of the first one."""
+    q, s, x = case(31 + M + K, M, N, K, bits, group)
+    desc = P.Desc(N, K, bits, group)
+    blob = torch.from_numpy(P.qlinear_pack(desc, q, s)).cuda()
+    lins = [P.QLinear(desc, blob), P.QLinear(desc, blob.clone())]
+    xd = torch.from_numpy(x).cuda()
+    y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    first = lins[0].forward(xd).clone()
+    for rnd in range(6):
+        for i in range(400):
+            lins[i & 1].forward_raw(xd.data_ptr(), y.data_ptr(), M)
+        assert torch.equal(y.view(torch.int16), first.view(torch.int16)), f"round {rnd}"
+    torch.cuda.synchronize()
+    assert lins[0].device_status() == (0, 0)
