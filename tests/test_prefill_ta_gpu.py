@@ -165,3 +165,35 @@ def test_back_to_back_launches_keep_their_bits(P, torch, M, N, K, bits, group):
         assert torch.equal(y.view(torch.int16), first.view(torch.int16)), f"round {rnd}"
     torch.cuda.synchronize()
     assert lins[0].device_status() == (0, 0)
+
+
+@pytest.mark.parametrize("form", ["gated", "grouped", "gated_fallback"])
+def test_back_to_back_multi_layer_launches_keep_their_bits(P, torch, form):
+    """The same for the launches that serve two layers: the fused gating (gate tile and up tile of a position back to
+    back in one cluster), the grouped launch, and the gating of a shape the fused kernel does not take (both
+    projections into the device scratch, then the element-wise kernel)."""
+    M, N, K = (2048, 9728, 1024) if form != "gated_fallback" else (96, 2304, 2048)
+    lins, xs = [], None
+    for i in range(2):
+        q, s, x = case(53 + i, M, N, K, 4, 32)
+        desc = P.Desc(N, K, 4, 32)
+        lins.append(P.QLinear(desc, torch.from_numpy(P.qlinear_pack(desc, q, s)).cuda()))
+        xs = x
+    xd = torch.from_numpy(xs).cuda()
+    ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _ in range(2)]
+
+    def launch():
+        if form == "grouped":
+            P.qlinear_forward_group_raw(lins, xd.data_ptr(), [y.data_ptr() for y in ys], M)
+        else:
+            P.qlinear_forward_gated_raw(lins[0], lins[1], xd.data_ptr(), ys[0].data_ptr(), M, "silu")
+    launch()
+    first = [y.clone() for y in ys]
+    n_out = 2 if form == "grouped" else 1
+    for rnd in range(5):
+        for _ in range(300):
+            launch()
+        for y, f in zip(ys[:n_out], first[:n_out]):
+            assert torch.equal(y.view(torch.int16), f.view(torch.int16)), f"round {rnd}"
+    torch.cuda.synchronize()
+    assert lins[0].device_status() == (0, 0)
