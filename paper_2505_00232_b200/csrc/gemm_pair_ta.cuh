@@ -530,13 +530,17 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                             orow[(cc + 4 * v4 + 3) * 128] = __float2half_rn(f.w * (scale * (float)((int)r[4 * v4 + 3] - OFF * i.w)));
                         }
                     } else if (!(QL_TA_EXP & 2)) {
+                        // (the kind of activation is chosen outside the element loop: inside it, the compiler evaluates
+                        // every kind and selects)
+                        auto store32 = [&](auto f) {
 #pragma unroll
-                        for (int q = 0; q < 32; ++q) {
-                            float v = __uint_as_float(r[q]) * scale;
-                            if (GATED && gl == 0) v = gate_activation(v, p.act);
-                            if (GATED && gl == 1) v *= __half2float(orow[(cc + q) * 128]);   // this thread's own act(gate)
-                            orow[(cc + q) * 128] = __float2half_rn(v);
-                        }
+                            for (int q = 0; q < 32; ++q) orow[(cc + q) * 128] = __float2half_rn(f(__uint_as_float(r[q]) * scale, q));
+                        };
+                        if (!GATED) store32([](float v, int) { return v; });
+                        else if (gl == 1) store32([&](float v, int q) { return v * __half2float(orow[(cc + q) * 128]); });   // this thread's own act(gate)
+                        else if (p.act == QL_ACT_SILU) store32([](float v, int) { return gate_activation(v, QL_ACT_SILU); });
+                        else if (p.act == QL_ACT_GELU_TANH) store32([](float v, int) { return gate_activation(v, QL_ACT_GELU_TANH); });
+                        else store32([](float v, int) { return v; });
                     }
                 }
                 fence_async_smem();
