@@ -118,24 +118,24 @@ ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int d
 ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
 
 /* The same result as n calls of qlinear_forward with one x: ys_dev[i] = x . W_i^T for the n layers hs[i]
- * (1 <= n <= 4), which must live on one device and agree in K, bits and group (q/k/v projections; gate
+ * (1 <= n <= 8), which must live on one device and agree in K, bits and group (q/k/v projections; gate
  * and up projections).  For M <= 8 all n layers run in ONE decode kernel launch: their output channels
  * are numbered one after the other and spread over the grid together, so short layers do not each pay
  * a launch of their own (the paper's operator fusion, Section 3 "Operator Fusion", merges kernels for
  * the same reason: launch overhead and memory-bound work).  Every output is bit-identical to what
  * qlinear_forward gives for that layer only if the K split chosen for the group equals the layer's own;
  * it always meets the same tolerance, and is run-to-run deterministic.  For larger M the layers share
- * one launch of the prefill kernel when every layer qualifies for its CTA-pair form (M > 128 and a
- * multiple of 256 output channels after padding to 128); the tiles of all layers then fill the
- * persistent grid together.  Otherwise they run one after the other.
+ * one launch of the prefill kernel when there are at most 4 of them and every layer qualifies for its
+ * CTA-pair form (a multiple of 256 output channels after padding to 128); the tiles of all layers then
+ * fill the persistent grid together.  Otherwise they run one after the other.
  *   hs      host array of n handles; ys_dev host array of n device pointers (fp16 [M, N_i], 16-byte
  *           aligned, not overlapping x_dev or one another); x_dev as in qlinear_forward.
  * Asynchronous, allocates nothing; the plan of the group is made per call and nothing is written to a handle.
- * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..4 or layers that do not agree. */
+ * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..8 or layers that do not agree. */
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
 
-/* Layers with DIFFERENT inputs in one launch: ys[i] = xs[i] . W_i^T for i < n (1 <= n <= 4), all with the same M.  The
+/* Layers with DIFFERENT inputs in one launch: ys[i] = xs[i] . W_i^T for i < n (1 <= n <= 8), all with the same M.  The
  * case in mind is the attention products over the KV cache held as weights (paper Section 3.8): every KV head has its
  * own cache handle and its own query rows, and a launch per head and product is launch-bound.  Same requirements on the
  * handles as qlinear_forward_group (one device, equal K, bits and group).  For M <= 8 and K a whole number of chunks the
@@ -211,7 +211,9 @@ ql_status qlinear_quantize_activations(const void* x_dev, int8_t* xq_dev, float*
  * These are the only calls that write to a blob; they must be ordered against forward calls on the same handles.
  * qlinear_kv_scores:  scores_dev [R, cache positions] = q_rows_dev [R, d_h] . K^T   (= qlinear_forward on h_k).
  * qlinear_kv_output:  out_dev [R, d_h] from prob_dev fp16 [R, cache positions]; tmp_dev is caller-owned scratch of
- *                     the same shape as prob_dev (it receives prob * s_v rounded to fp16).
+ *                     the same shape as prob_dev (it receives prob * s_v rounded to fp16 where that product needs a
+ *                     pass of its own: R > 8, or a cache length that is not a multiple of 32).
+ * k_new_dev, v_new_dev, v_scale_dev, prob_dev, tmp_dev, out_dev: 16-byte aligned.
  * Masking and the softmax between the two are the caller's.  Asynchronous, allocate nothing.
  * Errors: QL_ERR_INVALID_ARG (null / misaligned pointers, handles that are not an int8 cache pair of matching
  * shape, pos + n_new beyond the cache, d_h > 1024), otherwise as qlinear_forward. */
@@ -220,6 +222,29 @@ ql_status qlinear_kv_append(qlinear_t h_k, qlinear_t h_v, const void* k_new_dev,
 ql_status qlinear_kv_scores(qlinear_t h_k, const void* q_rows_dev, void* scores_dev, int32_t R, void* cuda_stream);
 ql_status qlinear_kv_output(qlinear_t h_v, const void* prob_dev, const void* v_scale_dev, void* tmp_dev, void* out_dev,
                             int32_t R, void* cuda_stream);
+
+/* The same three steps for ALL KV heads of an attention layer at once (n_heads <= 16 cache pairs of equal shape, arrays
+ * of handles h_k[i], h_v[i] and of their scale arrays v_scale_dev[i], all host arrays of device pointers): one launch per
+ * step for up to 8 heads instead of one (or two) per head -- at decode every one of these products is a few hundred
+ * KB and bound by the launch, not by the bytes.  The buffers have the layout the rotary / layout kernel writes:
+ *   qlinear_kv_append_heads: element (head i, new token t, dimension j) of k_new_dev / v_new_dev at
+ *                            i * head_stride + t * token_stride + j (strides in elements, multiples of 8;
+ *                            k_out / v_out of qlinear_rope_qkv: head_stride = S * d_h, token_stride = d_h)
+ *   qlinear_kv_scores_heads: q_rows_dev fp16 [n_heads, R, d_h] -> scores_dev fp16 [n_heads, R, cache positions]
+ *   qlinear_kv_output_heads: prob_dev fp16 [n_heads, R, cache positions] -> out_dev fp16 [n_heads, R, d_h]; R <= 8 and
+ *                            a cache length that is a multiple of 32: the product prob * s_v (rounded to fp16, as in
+ *                            qlinear_kv_output) is formed inside the decode kernel on the way to the tensor core, so
+ *                            there is no scratch buffer and no pass of its own.  Other shapes: QL_ERR_UNSUPPORTED
+ *                            (use qlinear_kv_output per head).
+ * All device pointers 16-byte aligned, R * d_h and R * cache positions multiples of 8.  Results are bit-identical to
+ * the per-head calls.  Asynchronous, allocate nothing.  Errors as above. */
+ql_status qlinear_kv_append_heads(const qlinear_t* h_k, const qlinear_t* h_v, int32_t n_heads, const void* k_new_dev,
+                                  const void* v_new_dev, int64_t head_stride, int64_t token_stride, void* const* v_scale_dev,
+                                  int32_t pos, int32_t n_new, void* cuda_stream);
+ql_status qlinear_kv_scores_heads(const qlinear_t* h_k, int32_t n_heads, const void* q_rows_dev, void* scores_dev, int32_t R,
+                                  void* cuda_stream);
+ql_status qlinear_kv_output_heads(const qlinear_t* h_v, int32_t n_heads, const void* prob_dev, const void* const* v_scale_dev,
+                                  void* out_dev, int32_t R, void* cuda_stream);
 
 /* Embedding lookup from a quantised table (Section 4.2: the mixed 8/4/4 scheme keeps the embedding table
  * in int4 like the feed-forward weights).  The handle's layer is read as a table of N rows of K values:

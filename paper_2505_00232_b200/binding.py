@@ -22,7 +22,7 @@ QL_ACT_IDENTITY, QL_ACT_SILU, QL_ACT_GELU_TANH = 0, 1, 2
 ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL_ACT_GELU_TANH}
 
 EXPORTS = (
-    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_batch", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
+    "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_batch", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_kv_append_heads", "qlinear_kv_scores_heads", "qlinear_kv_output_heads", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
     "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
@@ -84,6 +84,13 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_rope_qkv.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
     lib.qlinear_debug_expire_wait.restype = ctypes.c_int
+    pvp = ctypes.POINTER(ctypes.c_void_p)
+    lib.qlinear_kv_append_heads.argtypes = [pvp, pvp, ctypes.c_int32, vp, vp, ctypes.c_int64, ctypes.c_int64, pvp, ctypes.c_int32, ctypes.c_int32, vp]
+    lib.qlinear_kv_append_heads.restype = ctypes.c_int
+    lib.qlinear_kv_scores_heads.argtypes = [pvp, ctypes.c_int32, vp, vp, ctypes.c_int32, vp]
+    lib.qlinear_kv_scores_heads.restype = ctypes.c_int
+    lib.qlinear_kv_output_heads.argtypes = [pvp, ctypes.c_int32, vp, pvp, vp, ctypes.c_int32, vp]
+    lib.qlinear_kv_output_heads.restype = ctypes.c_int
     lib.qlinear_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.qlinear_device_status.restype = ctypes.c_int
     lib.qlinear_decode_static.argtypes = [dp, vp, vp, vp, i32, ctypes.c_int, vp]
@@ -205,7 +212,7 @@ def qlinear_forward_batch_raw(lins, x_ptrs, y_ptrs, M: int, stream=None) -> None
 
 
 def qlinear_forward_batch(lins, xs, outs=None, stream=None):
-    """xs: one fp16 CUDA tensor [M, K] per layer -> list of fp16 [M, N_i] (one launch for M <= 8, up to 4 layers)."""
+    """xs: one fp16 CUDA tensor [M, K] per layer -> list of fp16 [M, N_i] (one launch for M <= 8, up to 8 layers)."""
     import torch
     K, M = lins[0].desc.K, xs[0].shape[0]
     if len(xs) != len(lins):
@@ -223,7 +230,7 @@ def qlinear_forward_batch(lins, xs, outs=None, stream=None):
 
 
 def kv_scores_batch(caches, q_rows, stream=None):
-    """The score product of up to 4 KV heads in one launch: caches[i].scores(q_rows[i]) for every i (paper Section 3.8)."""
+    """The score product of up to 8 KV heads in one launch: caches[i].scores(q_rows[i]) for every i (paper Section 3.8)."""
     return qlinear_forward_batch([c.k for c in caches], q_rows, stream=stream)
 
 
@@ -472,4 +479,61 @@ class KVCache:
         _check(lib.qlinear_kv_output(self.v._h, ctypes.c_void_p(prob.data_ptr()), ctypes.c_void_p(self.v_scale.data_ptr()),
                                      ctypes.c_void_p(tmp.data_ptr()), ctypes.c_void_p(out.data_ptr()), prob.shape[0], _stream_ptr(stream)),
                "qlinear_kv_output")
+        return out
+
+
+class KVHeads:
+    """The caches of all KV heads of one attention layer (n_heads <= 16 KVCache objects of equal shape), driven through
+    the calls that serve every head in one launch (qlinear_kv_*_heads in include/qlinear.h): argument marshalling only."""
+
+    def __init__(self, n_heads: int, cache_size: int, d_h: int, device="cuda:0"):
+        self.heads = [KVCache(cache_size, d_h, device) for _ in range(n_heads)]
+        self.n, self.cache_size, self.d_h, self.length = n_heads, cache_size, d_h, 0
+        arr = ctypes.c_void_p * n_heads
+        self._hk = arr(*[c.k._h for c in self.heads])
+        self._hv = arr(*[c.v._h for c in self.heads])
+        self._vs = arr(*[ctypes.c_void_p(c.v_scale.data_ptr()) for c in self.heads])
+
+    def append_raw(self, k_ptr: int, v_ptr: int, head_stride: int, token_stride: int, n_new: int, stream=None) -> None:
+        _check(lib.qlinear_kv_append_heads(self._hk, self._hv, self.n, ctypes.c_void_p(k_ptr), ctypes.c_void_p(v_ptr), head_stride, token_stride,
+                                           self._vs, self.length, n_new, _stream_ptr(stream)), "qlinear_kv_append_heads")
+        self.length += n_new
+        for c in self.heads:
+            c.length = self.length
+
+    def append(self, k_new, v_new, stream=None):
+        """k_new, v_new: fp16 CUDA [n_heads, n_new, d_h] (the k_out / v_out of qlinear_rope_qkv)."""
+        import torch
+        for t in (k_new, v_new):
+            if t.dim() != 3 or t.shape[0] != self.n or t.shape[2] != self.d_h or t.dtype != torch.float16 or not t.is_cuda or not t.is_contiguous():
+                raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_append_heads (k_new, v_new must be contiguous fp16 CUDA [n_heads, n_new, d_h])")
+        if k_new.shape != v_new.shape:
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_append_heads (k_new and v_new differ in shape)")
+        n_new = k_new.shape[1]
+        self.append_raw(k_new.data_ptr(), v_new.data_ptr(), n_new * self.d_h, self.d_h, n_new, stream)
+
+    def scores_raw(self, q_ptr: int, out_ptr: int, R: int, stream=None) -> None:
+        _check(lib.qlinear_kv_scores_heads(self._hk, self.n, ctypes.c_void_p(q_ptr), ctypes.c_void_p(out_ptr), R, _stream_ptr(stream)),
+               "qlinear_kv_scores_heads")
+
+    def scores(self, q_rows, stream=None):
+        """q_rows fp16 [n_heads, R, d_h] -> fp16 [n_heads, R, cache_size]."""
+        import torch
+        if q_rows.dim() != 3 or q_rows.shape[0] != self.n or q_rows.shape[2] != self.d_h or q_rows.dtype != torch.float16 or not q_rows.is_cuda or not q_rows.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_scores_heads (q_rows must be contiguous fp16 CUDA [n_heads, R, d_h])")
+        out = torch.empty((self.n, q_rows.shape[1], self.cache_size), dtype=torch.float16, device=q_rows.device)
+        self.scores_raw(q_rows.data_ptr(), out.data_ptr(), q_rows.shape[1], stream)
+        return out
+
+    def output_raw(self, prob_ptr: int, out_ptr: int, R: int, stream=None) -> None:
+        _check(lib.qlinear_kv_output_heads(self._hv, self.n, ctypes.c_void_p(prob_ptr), self._vs, ctypes.c_void_p(out_ptr), R, _stream_ptr(stream)),
+               "qlinear_kv_output_heads")
+
+    def output(self, prob, stream=None):
+        """prob fp16 [n_heads, R, cache_size] -> fp16 [n_heads, R, d_h]."""
+        import torch
+        if prob.dim() != 3 or prob.shape[0] != self.n or prob.shape[2] != self.cache_size or prob.dtype != torch.float16 or not prob.is_cuda or not prob.is_contiguous():
+            raise QLinearError(QL_ERR_INVALID_ARG, "qlinear_kv_output_heads (prob must be contiguous fp16 CUDA [n_heads, R, cache_size])")
+        out = torch.empty((self.n, prob.shape[1], self.d_h), dtype=torch.float16, device=prob.device)
+        self.output_raw(prob.data_ptr(), out.data_ptr(), prob.shape[1], stream)
         return out

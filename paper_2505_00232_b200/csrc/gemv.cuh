@@ -28,7 +28,7 @@ constexpr int kGemvWarps = 8;
 constexpr int kGemvThreads = kGemvWarps * 32;
 constexpr int kGemvRing = 8;             // chunks prefetched per warp (cp.async ring slots)
 
-constexpr int kGemvMaxGroup = 4;         // layers that may share one launch (same input, same K and scheme)
+constexpr int kGemvMaxGroup = 8;         // layers that may share one launch (same K and scheme)
 
 struct GemvParams {
     // One launch serves up to kGemvMaxGroup layers that read the same x (q/k/v, gate/up): their row-blocks
@@ -43,6 +43,10 @@ struct GemvParams {
     // Batched form (layers with DIFFERENT inputs in one launch, e.g. the score products of several KV heads): the input
     // of layer i; the plain and grouped forms set every entry to x.  Only the direct form (XDIRECT) reads it per layer.
     const __half* xl[kGemvMaxGroup];
+    // XSCALE form (the V-cache product of paper Section 3.8): layer i's input is multiplied element-wise by the fp16 vector
+    // xscale[i][0 .. K) on its way to the tensor core (x'[m, k] = fp16(x[m, k] * xscale[k])): the per-token scales of a
+    // value cache folded into the attention probabilities without a pass of their own.
+    const __half* xscale[kGemvMaxGroup];
     int32_t M, K;
     int32_t n_rb;                        // row-blocks holding at least one real row, all layers
     int32_t n_kc;                        // chunks along K
@@ -60,7 +64,7 @@ struct GemvParams {
 // alternately, so that a CTA (which then holds an even number of row-blocks, no cluster) has both branches of
 // every output channel it owns; the epilogue writes y[0] = act(gate) * up (paper Section 3.6: element-wise
 // operators of two branches fused with a fully connected operator).
-template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false>
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false>
 __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -150,6 +154,18 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     // independent and those columns are never stored.
     const __half* xpass = XDIRECT ? p.xl[layer] + (int64_t)min(g, p.M - 1) * p.K + 8 * c + kc0 * CHUNK_K
                                   : xs + min(g, p.M - 1) * p.x_stride + 8 * c + (kc0 * CHUNK_K - k_cta0);
+    static_assert(!XSCALE || (XDIRECT && BITS == 8 && !GATED), "the scaled-input form exists for int8 layers read straight from global memory");
+    const __half* spass = XSCALE ? p.xscale[layer] + 8 * c + kc0 * CHUNK_K : nullptr;
+    auto scale_x = [](uint4 v, const __half* sptr) {                     // fp16 products, one rounding each
+        const uint4 sv = *reinterpret_cast<const uint4*>(sptr);
+        const __half2* a = reinterpret_cast<const __half2*>(&v);
+        const __half2* b = reinterpret_cast<const __half2*>(&sv);
+        uint4 r;
+        __half2* o = reinterpret_cast<__half2*>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i] = __hmul2(a[i], b[i]);
+        return r;
+    };
     // Direct form: the host chooses it only when K is a whole number of chunks, so every chunk in
     // [kc0, kc1) lies inside the token's row and the loads need no bounds check.
     auto load_x = [&](const __half* ptr) {
@@ -222,7 +238,11 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
             // x fragments first: their latency (L1 / shared) runs under the wait for the weights
             const __half* xk = xpass + d * CHUNK_K;
             const __half* xk1 = two ? xk + CHUNK_K : xk;                 // odd tail: stay inside the row
-            const uint4 x00 = load_x(xk), x10 = load_x(xk1);
+            uint4 x00 = load_x(xk), x10 = load_x(xk1);
+            if (XSCALE) {
+                x00 = scale_x(x00, spass + d * CHUNK_K);
+                x10 = scale_x(x10, spass + (two ? d + 1 : d) * CHUNK_K);
+            }
             uint4 x01 = x00, x11 = x10;
             if (BITS == 4) { x01 = load_x(xk + 32); x11 = load_x(xk1 + 32); }
             asm volatile("cp.async.wait_group %0;" ::"n"(kGemvRing / 2 - 1) : "memory");
@@ -255,6 +275,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
         if (BITS == 8 && kc + 2 * kGemvRing <= kc1) pass(false, kc);
         else pass(true, kc);
         xpass += kGemvRing * CHUNK_K;
+        if (XSCALE) spass += kGemvRing * CHUNK_K;
         sflip ^= 1;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");

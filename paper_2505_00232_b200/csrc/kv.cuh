@@ -28,25 +28,31 @@ __host__ __device__ __forceinline__ int64_t int8_weight_offset(int row, int k, i
     return ((int64_t)rsb * n_kc + kc) * kWeightBlockBytes + rb * 512 + ((g << 2) | c) * 16 + w * 4 + b;
 }
 
+constexpr int kKvMaxHeads = 16;          // KV heads (cache pairs of equal shape) that one append launch serves
+
 struct KvAppendParams {
-    uint8_t* k_body;         // K cache: N = cache positions, K = d_h
-    __half* k_scales;        // its per-channel (= per-token) scales
-    uint8_t* v_body;         // V cache: N = d_h, K = cache positions
-    __half* v_scale;         // [cache positions] per-token scales of V (side array)
-    const __half* k_new;     // [n_new, d_h]
-    const __half* v_new;     // [n_new, d_h]
+    // per head (blockIdx.y)
+    uint8_t* k_body[kKvMaxHeads];        // K cache: N = cache positions, K = d_h
+    __half* k_scales[kKvMaxHeads];       // its per-channel (= per-token) scales
+    uint8_t* v_body[kKvMaxHeads];        // V cache: N = d_h, K = cache positions
+    __half* v_scale[kKvMaxHeads];        // [cache positions] per-token scales of V (side array)
+    const __half* k_new;                 // element (head h, new token i, dimension j) at h * head_stride + i * token_stride + j
+    const __half* v_new;
+    int64_t head_stride, token_stride;
     int32_t d_h, cache_size, pos, n_new;
     int32_t k_n_kc, v_n_kc;
 };
 
-// One CTA (128 threads) per new token; d_h <= 1024.
+// One CTA (128 threads) per new token and head; d_h <= 1024.
 __global__ void __launch_bounds__(128) kv_append_kernel(const KvAppendParams p)
 {
     __shared__ float wmax[2][4];
     __shared__ float sc[2];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int i = blockIdx.x, t = p.pos + i;
-    const __half* kv[2] = {p.k_new + (int64_t)i * p.d_h, p.v_new + (int64_t)i * p.d_h};
+    const int i = blockIdx.x, t = p.pos + i, hd = blockIdx.y;
+    const int64_t src = hd * p.head_stride + i * p.token_stride;
+    const __half* kv[2] = {p.k_new + src, p.v_new + src};
     float am[2] = {0.f, 0.f};
     for (int j = threadIdx.x; j < p.d_h; j += 128) {
         am[0] = fmaxf(am[0], fabsf(__half2float(kv[0][j])));
@@ -66,7 +72,7 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const KvAppendParams p)
         const bool dead = __half2float(h0) == 0.f;                       // a zero vector, or a scale below fp16's range
         sc[s] = dead ? 0.f : __half2float(h0);                           // 0 marks "store zeros"
         const __half h = dead ? __float2half_rn(1.f) : h0;
-        if (s == 0) p.k_scales[t] = h; else p.v_scale[t] = h;
+        if (s == 0) p.k_scales[hd][t] = h; else p.v_scale[hd][t] = h;
     }
     __syncthreads();
     for (int j = threadIdx.x; j < p.d_h; j += 128) {
@@ -75,8 +81,8 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const KvAppendParams p)
             int q = 0;
             if (sc[s] != 0.f) q = max(-127, min(127, __float2int_rn(__fdiv_rn(__half2float(kv[s][j]), sc[s]))));
             const uint8_t stored = (uint8_t)(q + 128);
-            if (s == 0) p.k_body[int8_weight_offset(t, j, p.k_n_kc)] = stored;      // K: row = token, k = dimension
-            else p.v_body[int8_weight_offset(j, t, p.v_n_kc)] = stored;             // V: row = dimension, k = token
+            if (s == 0) p.k_body[hd][int8_weight_offset(t, j, p.k_n_kc)] = stored;  // K: row = token, k = dimension
+            else p.v_body[hd][int8_weight_offset(j, t, p.v_n_kc)] = stored;         // V: row = dimension, k = token
         }
     }
 }

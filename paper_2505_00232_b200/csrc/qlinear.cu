@@ -224,19 +224,22 @@ cudaError_t ensure_smem_attr(Kern kern, std::atomic<bool>* flags, int device, in
     return e;
 }
 
-template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false>
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false>
 cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
 {
     static std::atomic<bool> attr_set[kMaxDevices];
-    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT, GATED>;
+    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT, GATED, XSCALE>;
     cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, kGemvMaxSmem);
     if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
 }
 
 template <int BITS, bool GROUPED>
-cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st, bool gated = false)
+cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st, bool gated = false, bool xscale = false)
 {
+    if constexpr (BITS == 8 && !GROUPED) {
+        if (xscale) return launch_gemv_x<8, false, true, false, true>(h, prm, pl, st);   // (int8, direct x: checked by the caller)
+    }
     if (gated) return launch_gemv_x<BITS, GROUPED, true, true>(h, prm, pl, st);     // (planned only with direct x)
     return prm.x_bytes == 0 ? launch_gemv_x<BITS, GROUPED, true>(h, prm, pl, st)
                             : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
@@ -246,9 +249,9 @@ cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPla
 // call (integer arithmetic only); nothing is written to a handle.
 // act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
 // xs != nullptr: the batched form, layer i reads xs[i] (x is then ignored); needs the kernel form that reads x straight
-// from global memory.
+// from global memory.  xscales != nullptr (with xs, int8 layers): layer i's input is multiplied by xscales[i][0 .. K).
 ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1,
-                       const void* const* xs = nullptr)
+                       const void* const* xs = nullptr, const void* const* xscales = nullptr)
 {
     const qlinear_s* h = hs[0];
     const Layout& L = h->L;
@@ -258,6 +261,7 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     if (gated) n_rb = 2 * hs[0]->n_rb;
     const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
     if ((gated || xs) && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
+    if (xscales && (!xs || L.bits != 8)) return QL_ERR_UNSUPPORTED;
     cudaError_t e;
     if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
     GemvParams prm{};
@@ -274,13 +278,16 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     prm.n_layers = n;
     prm.act = gated ? act : 0;
     prm.x = static_cast<const __half*>(xs ? xs[0] : x);
-    for (int i = 0; i < kGemvMaxGroup; ++i) prm.xl[i] = static_cast<const __half*>(xs ? xs[i < n ? i : 0] : x);
+    for (int i = 0; i < kGemvMaxGroup; ++i) {
+        prm.xl[i] = static_cast<const __half*>(xs ? xs[i < n ? i : 0] : x);
+        prm.xscale[i] = static_cast<const __half*>(xscales ? xscales[i < n ? i : 0] : nullptr);
+    }
     prm.M = M; prm.K = L.K;
     prm.n_rb = n_rb;
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
-    if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st, gated);
+    if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st, gated, xscales != nullptr);
     else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st, gated);
     else e = launch_gemv<4, false>(h, prm, pl, st, gated);
     return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
@@ -539,7 +546,7 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
         return forward_gemv(const_cast<qlinear_s* const*>(hs), n, x, ys, M, static_cast<cudaStream_t>(stream));
     }
-    if (n > 1 && M > hs[0]->gemv_max_m) {                                // prefill: one launch of the CTA-pair kernel
+    if (n > 1 && n <= kGemmMaxGroup && M > hs[0]->gemv_max_m) {          // prefill: one launch of the CTA-pair kernel
         bool pair_ok = true;
         for (int i = 0; i < n; ++i) pair_ok = pair_ok && (hs[i]->L.n_rsb % 2) == 0 && (gemm_pair_applicable(hs[i]->L, M) || (hs[i]->wmap_ok && gemm_config().ta));
         if (pair_ok) {
@@ -701,30 +708,47 @@ extern "C" ql_status qlinear_quantize_activations(const void* x, int8_t* xq, flo
     return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
 }
 
+extern "C" ql_status qlinear_kv_append_heads(const qlinear_t* hk, const qlinear_t* hv, int32_t n_heads, const void* k_new, const void* v_new,
+                                             int64_t head_stride, int64_t token_stride, void* const* v_scales, int32_t pos, int32_t n_new,
+                                             void* stream)
+{
+    if (!hk || !hv || !v_scales || n_heads < 1 || n_heads > kKvMaxHeads || !k_new || !v_new || pos < 0 || n_new < 0) return QL_ERR_INVALID_ARG;
+    if (head_stride < 0 || token_stride < 0 || ((head_stride | token_stride) & 7)) return QL_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) & 15) return QL_ERR_INVALID_ARG;
+    for (int i = 0; i < n_heads; ++i) {
+        if (!hk[i] || !hv[i] || !v_scales[i] || (reinterpret_cast<uintptr_t>(v_scales[i]) & 15)) return QL_ERR_INVALID_ARG;
+        const Layout &K = hk[i]->L, &V = hv[i]->L;
+        if (hk[i]->device != hk[0]->device || hv[i]->device != hk[0]->device) return QL_ERR_INVALID_ARG;
+        if (K.bits != 8 || V.bits != 8 || K.N != V.K || K.K != V.N || K.N != hk[0]->L.N || K.K != hk[0]->L.K) return QL_ERR_INVALID_ARG;
+    }
+    const Layout &K = hk[0]->L, &V = hv[0]->L;
+    if ((int64_t)pos + n_new > K.N || K.K > 1024) return QL_ERR_INVALID_ARG;
+    if (n_new == 0) return QL_OK;
+    DeviceGuard guard(hk[0]->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    KvAppendParams prm{};
+    for (int i = 0; i < n_heads; ++i) {
+        uint8_t* kb = const_cast<uint8_t*>(hk[i]->blob);                 // the caches are the one kind of blob the library writes
+        uint8_t* vb = const_cast<uint8_t*>(hv[i]->blob);
+        prm.k_body[i] = kb + K.body_offset;
+        prm.k_scales[i] = reinterpret_cast<__half*>(kb + K.chan_scale_offset);
+        prm.v_body[i] = vb + V.body_offset;
+        prm.v_scale[i] = static_cast<__half*>(v_scales[i]);
+    }
+    prm.k_new = static_cast<const __half*>(k_new);
+    prm.v_new = static_cast<const __half*>(v_new);
+    prm.head_stride = head_stride; prm.token_stride = token_stride;
+    prm.d_h = K.K; prm.cache_size = K.N; prm.pos = pos; prm.n_new = n_new;
+    prm.k_n_kc = K.n_kc; prm.v_n_kc = V.n_kc;
+    const cudaError_t e = launch(kv_append_kernel, prm, dim3(n_new, n_heads), dim3(128), 0, static_cast<cudaStream_t>(stream), 1, hk[0]->pdl);
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
 extern "C" ql_status qlinear_kv_append(qlinear_t hk, qlinear_t hv, const void* k_new, const void* v_new, void* v_scale,
                                        int32_t pos, int32_t n_new, void* stream)
 {
-    if (!hk || !hv || !k_new || !v_new || !v_scale || pos < 0 || n_new < 0) return QL_ERR_INVALID_ARG;
-    const Layout &K = hk->L, &V = hv->L;
-    if (hk->device != hv->device || K.bits != 8 || V.bits != 8 || K.N != V.K || K.K != V.N) return QL_ERR_INVALID_ARG;
-    if ((int64_t)pos + n_new > K.N || K.K > 1024) return QL_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new) | reinterpret_cast<uintptr_t>(v_scale)) & 1) return QL_ERR_INVALID_ARG;
-    if (n_new == 0) return QL_OK;
-    DeviceGuard guard(hk->device);
-    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
-    KvAppendParams prm{};
-    uint8_t* kb = const_cast<uint8_t*>(hk->blob);                        // the caches are the one kind of blob the library writes
-    uint8_t* vb = const_cast<uint8_t*>(hv->blob);
-    prm.k_body = kb + K.body_offset;
-    prm.k_scales = reinterpret_cast<__half*>(kb + K.chan_scale_offset);
-    prm.v_body = vb + V.body_offset;
-    prm.v_scale = static_cast<__half*>(v_scale);
-    prm.k_new = static_cast<const __half*>(k_new);
-    prm.v_new = static_cast<const __half*>(v_new);
-    prm.d_h = K.K; prm.cache_size = K.N; prm.pos = pos; prm.n_new = n_new;
-    prm.k_n_kc = K.n_kc; prm.v_n_kc = V.n_kc;
-    kv_append_kernel<<<n_new, 128, 0, static_cast<cudaStream_t>(stream)>>>(prm);
-    return cudaGetLastError() == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+    if (!hk || !hv) return QL_ERR_INVALID_ARG;
+    return qlinear_kv_append_heads(&hk, &hv, 1, k_new, v_new, 0, hk->L.K, &v_scale, pos, n_new, stream);
 }
 
 extern "C" ql_status qlinear_kv_scores(qlinear_t hk, const void* q_rows, void* scores, int32_t R, void* stream)
@@ -733,12 +757,68 @@ extern "C" ql_status qlinear_kv_scores(qlinear_t hk, const void* q_rows, void* s
     return qlinear_forward(hk, q_rows, scores, R, stream);
 }
 
+extern "C" ql_status qlinear_kv_scores_heads(const qlinear_t* hk, int32_t n_heads, const void* q_rows, void* scores, int32_t R, void* stream)
+{
+    if (!hk || n_heads < 1 || n_heads > kKvMaxHeads || !q_rows || !scores || R < 1) return QL_ERR_INVALID_ARG;
+    for (int i = 0; i < n_heads; ++i)
+        if (!hk[i] || hk[i]->L.bits != 8 || hk[i]->L.N != hk[0]->L.N || hk[i]->L.K != hk[0]->L.K) return QL_ERR_INVALID_ARG;
+    const int64_t xs_stride = (int64_t)R * hk[0]->L.K, ys_stride = (int64_t)R * hk[0]->L.N;
+    if ((xs_stride | ys_stride) & 7) return QL_ERR_INVALID_ARG;          // every head's rows start on a 16-byte boundary
+    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxGroup) {
+        const int n = std::min(kGemvMaxGroup, n_heads - h0);
+        const void* xs[kGemvMaxGroup];
+        void* ys[kGemvMaxGroup];
+        for (int i = 0; i < n; ++i) {
+            xs[i] = static_cast<const __half*>(q_rows) + (h0 + i) * xs_stride;
+            ys[i] = static_cast<__half*>(scores) + (h0 + i) * ys_stride;
+        }
+        const ql_status s = qlinear_forward_batch(hk + h0, n, xs, ys, R, stream);
+        if (s != QL_OK) return s;
+    }
+    return QL_OK;
+}
+
+extern "C" ql_status qlinear_kv_output_heads(const qlinear_t* hv, int32_t n_heads, const void* prob, const void* const* v_scales, void* out,
+                                             int32_t R, void* stream)
+{
+    if (!hv || !v_scales || n_heads < 1 || n_heads > kKvMaxHeads || !prob || !out || R < 1) return QL_ERR_INVALID_ARG;
+    for (int i = 0; i < n_heads; ++i) {
+        if (!hv[i] || !v_scales[i] || (reinterpret_cast<uintptr_t>(v_scales[i]) & 15)) return QL_ERR_INVALID_ARG;
+        if (hv[i]->L.bits != 8 || hv[i]->L.N != hv[0]->L.N || hv[i]->L.K != hv[0]->L.K || hv[i]->device != hv[0]->device) return QL_ERR_INVALID_ARG;
+    }
+    const Layout& V = hv[0]->L;
+    const int64_t xs_stride = (int64_t)R * V.K, ys_stride = (int64_t)R * V.N;
+    if ((xs_stride | ys_stride) & 7) return QL_ERR_INVALID_ARG;
+    if (((reinterpret_cast<uintptr_t>(prob) | reinterpret_cast<uintptr_t>(out)) & 15) || xs_stride > INT32_MAX) return QL_ERR_INVALID_ARG;
+    if (R > hv[0]->gemv_max_m || hv[0]->use_stream) return QL_ERR_UNSUPPORTED;          // the fused form exists in the decode kernel
+    if (device_timed_out(hv[0])) return QL_ERR_DEVICE_TIMEOUT;
+    DeviceGuard guard(hv[0]->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxGroup) {
+        const int n = std::min(kGemvMaxGroup, n_heads - h0);
+        const void* xs[kGemvMaxGroup];
+        void* ys[kGemvMaxGroup];
+        for (int i = 0; i < n; ++i) {
+            xs[i] = static_cast<const __half*>(prob) + (h0 + i) * xs_stride;
+            ys[i] = static_cast<__half*>(out) + (h0 + i) * ys_stride;
+        }
+        const ql_status s = forward_gemv(const_cast<qlinear_s* const*>(hv + h0), n, nullptr, ys, R, static_cast<cudaStream_t>(stream), -1, xs, v_scales + h0);
+        if (s != QL_OK) return s;
+    }
+    return QL_OK;
+}
+
 extern "C" ql_status qlinear_kv_output(qlinear_t hv, const void* prob, const void* v_scale, void* tmp, void* out, int32_t R, void* stream)
 {
     if (!hv || !prob || !v_scale || !tmp || !out || R < 1 || hv->L.bits != 8) return QL_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(tmp) | reinterpret_cast<uintptr_t>(out)) & 15) return QL_ERR_INVALID_ARG;
     const int T = hv->L.K;
     if ((int64_t)R * T > INT32_MAX) return QL_ERR_INVALID_ARG;
+    // decode-sized products whose cache length is a whole number of chunks: the scales are applied inside the kernel
+    if (!((reinterpret_cast<uintptr_t>(prob) | reinterpret_cast<uintptr_t>(v_scale)) & 15)) {
+        const ql_status s = qlinear_kv_output_heads(&hv, 1, prob, &v_scale, out, R, stream);
+        if (s != QL_ERR_UNSUPPORTED) return s;
+    }
     {
         DeviceGuard guard(hv->device);
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }

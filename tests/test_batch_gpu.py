@@ -90,4 +90,4 @@ def test_falls_back_for_prefill_sizes_and_checks_arguments(P, torch):
     with pytest.raises(P.QLinearError):
         P.qlinear_forward_batch(lins, xs[:1])
     with pytest.raises(P.QLinearError):
-        P.qlinear_forward_batch(lins * 3, xs * 3)                        # more than 4 layers
+        P.qlinear_forward_batch(lins * 5, xs * 5)                        # more than 8 layers

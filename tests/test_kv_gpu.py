@@ -88,3 +88,54 @@ def test_append_argument_errors(P, torch):
     import ctypes
     vp = ctypes.c_void_p
     assert P.lib.qlinear_kv_append(cache.k._h, other.v._h, vp(a.data_ptr()), vp(a.data_ptr()), vp(cache.v_scale.data_ptr()), 0, 1, None) == 1
+
+
+@pytest.mark.parametrize("n_heads", [3, 8, 11])
+def test_all_heads_in_one_launch_match_the_per_head_calls(P, torch, n_heads):
+    """qlinear_kv_*_heads (every KV head of a layer in one launch, value scales folded inside the decode kernel) against
+    the per-head calls: the same cache bytes and scales, the same score and output bits; and the output against the
+    oracle.  11 heads: more than one launch's worth."""
+    T, R = 1031, GROUP
+    ks, vs, qs = [], [], []
+    for h in range(n_heads):
+        k, v = tensors(1200 + h, T)
+        ks.append(k); vs.append(v); qs.append(gen.normal_fp16(1200 + h, 3, (R, DH)))
+    k_all, v_all, q_all = (torch.from_numpy(np.stack(a)).cuda() for a in (ks, vs, qs))
+    heads = P.KVHeads(n_heads, CACHE, DH)
+    heads.append(k_all[:, :1024].contiguous(), v_all[:, :1024].contiguous())        # prefill
+    for t in range(1024, T):                                                        # decode steps, strided input
+        heads.append_raw(k_all[:, t].data_ptr(), v_all[:, t].data_ptr(), T * DH, DH, 1)
+    singles = [P.KVCache(CACHE, DH) for _ in range(n_heads)]
+    for h, c in enumerate(singles):
+        c.append(k_all[h], v_all[h])
+    torch.cuda.synchronize()
+    assert heads.length == T
+    for h in range(n_heads):
+        assert torch.equal(heads.heads[h].k.packed, singles[h].k.packed)
+        assert torch.equal(heads.heads[h].v.packed, singles[h].v.packed)
+        assert torch.equal(heads.heads[h].v_scale, singles[h].v_scale)
+    sc = heads.scores(q_all)
+    z = sc[:, :, :T].double() / np.sqrt(DH)
+    prob = torch.zeros((n_heads, R, CACHE), dtype=torch.float16, device="cuda")
+    prob[:, :, :T] = torch.softmax(z, dim=2).half()
+    out = heads.output(prob)
+    torch.cuda.synchronize()
+    assert heads.heads[0].k.device_status() == (0, 0)
+    for h in range(n_heads):
+        assert torch.equal(sc[h], singles[h].scores(q_all[h]))
+        # the product with the scales as a pass of its own (one rounding to fp16), then the plain layer
+        folded = (prob[h].float() * singles[h].v_scale.float()[None, :]).half()
+        assert torch.equal(out[h], singles[h].v.forward(folded))
+        assert torch.equal(out[h], singles[h].output(prob[h]))
+        _, _, out64, A_out = O.kv_attention(qs[h], ks[h], vs[h], prob[h, :, :T].cpu().numpy())
+        ok, rel, worst = O.check_against(out[h].cpu().numpy(), out64, A_out)
+        assert ok, ("output", h, rel, worst)
+
+
+def test_heads_argument_errors(P, torch):
+    heads = P.KVHeads(2, 256, 64)
+    big = torch.zeros((2, 9, 256), dtype=torch.float16, device="cuda")
+    with pytest.raises(P.QLinearError):
+        heads.output(big)                               # 9 query rows: not a decode-sized product
+    with pytest.raises(P.QLinearError):
+        heads.append(torch.zeros((3, 1, 64), dtype=torch.float16, device="cuda"), torch.zeros((3, 1, 64), dtype=torch.float16, device="cuda"))
