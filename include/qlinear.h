@@ -118,20 +118,20 @@ ql_status qlinear_create(const qlinear_desc* desc, const void* packed_dev, int d
 ql_status qlinear_forward(qlinear_t h, const void* x_dev, void* y_dev, int32_t M, void* cuda_stream);
 
 /* The same result as n calls of qlinear_forward with one x: ys_dev[i] = x . W_i^T for the n layers hs[i]
- * (1 <= n <= 8), which must live on one device and agree in K, bits and group (q/k/v projections; gate
+ * (1 <= n <= 4), which must live on one device and agree in K, bits and group (q/k/v projections; gate
  * and up projections).  For M <= 8 all n layers run in ONE decode kernel launch: their output channels
  * are numbered one after the other and spread over the grid together, so short layers do not each pay
  * a launch of their own (the paper's operator fusion, Section 3 "Operator Fusion", merges kernels for
  * the same reason: launch overhead and memory-bound work).  Every output is bit-identical to what
  * qlinear_forward gives for that layer only if the K split chosen for the group equals the layer's own;
  * it always meets the same tolerance, and is run-to-run deterministic.  For larger M the layers share
- * one launch of the prefill kernel when there are at most 4 of them and every layer qualifies for its
+ * one launch of the prefill kernel when every layer qualifies for its
  * CTA-pair form (a multiple of 256 output channels after padding to 128); the tiles of all layers then
  * fill the persistent grid together.  Otherwise they run one after the other.
  *   hs      host array of n handles; ys_dev host array of n device pointers (fp16 [M, N_i], 16-byte
  *           aligned, not overlapping x_dev or one another); x_dev as in qlinear_forward.
  * Asynchronous, allocates nothing; the plan of the group is made per call and nothing is written to a handle.
- * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..8 or layers that do not agree. */
+ * Errors: as qlinear_forward; QL_ERR_INVALID_ARG also for n outside 1..4 or layers that do not agree. */
 ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_dev, void* const* ys_dev,
                                 int32_t M, void* cuda_stream);
 
@@ -139,7 +139,8 @@ ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const void* x_de
  * case in mind is the attention products over the KV cache held as weights (paper Section 3.8): every KV head has its
  * own cache handle and its own query rows, and a launch per head and product is launch-bound.  Same requirements on the
  * handles as qlinear_forward_group (one device, equal K, bits and group).  For M <= 8 and K a whole number of chunks the
- * call is one decode launch; otherwise it is n calls of qlinear_forward, in order.  Pointers as for qlinear_forward. */
+ * call is one decode launch (more than 4 layers: int8 layers only); otherwise it is n calls of qlinear_forward, in
+ * order.  Pointers as for qlinear_forward. */
 ql_status qlinear_forward_batch(const qlinear_t* handles, int32_t n, const void* const* xs_dev, void* const* ys_dev, int32_t M, void* cuda_stream);
 
 /* Activation of the gate branch in qlinear_forward_gated. */

@@ -212,7 +212,7 @@ def qlinear_forward_batch_raw(lins, x_ptrs, y_ptrs, M: int, stream=None) -> None
 
 
 def qlinear_forward_batch(lins, xs, outs=None, stream=None):
-    """xs: one fp16 CUDA tensor [M, K] per layer -> list of fp16 [M, N_i] (one launch for M <= 8, up to 8 layers)."""
+    """xs: one fp16 CUDA tensor [M, K] per layer -> list of fp16 [M, N_i] (one launch for M <= 8: up to 4 layers, 8 if they are int8)."""
     import torch
     K, M = lins[0].desc.K, xs[0].shape[0]
     if len(xs) != len(lins):

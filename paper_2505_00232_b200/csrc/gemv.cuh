@@ -28,25 +28,29 @@ constexpr int kGemvWarps = 8;
 constexpr int kGemvThreads = kGemvWarps * 32;
 constexpr int kGemvRing = 8;             // chunks prefetched per warp (cp.async ring slots)
 
-constexpr int kGemvMaxGroup = 8;         // layers that may share one launch (same K and scheme)
+constexpr int kGemvMaxGroup = 4;         // layers that may share one launch (same K and scheme)
+constexpr int kGemvMaxBatch = 8;         // ... in the form that serves the KV heads of an attention layer (NG = 8)
 
-struct GemvParams {
+// NG: capacity of the per-layer arrays.  The linear layers of a block come in groups of at most 4; the wider form is
+// a separate instantiation because the longer parameter block and layer searches cost the 4-layer launches about 1 %.
+template <int NG>
+struct GemvParamsT {
     // One launch serves up to kGemvMaxGroup layers that read the same x (q/k/v, gate/up): their row-blocks
     // are numbered one after the other; rb_end[i] is the number of row-blocks of layers 0..i.
-    const uint8_t* body[kGemvMaxGroup];  // first block of each packed body
-    const __half* chan_scales[kGemvMaxGroup];   // per-channel scales (nullptr when grouped)
-    __half* y[kGemvMaxGroup];            // [M, N_i]
-    int32_t N[kGemvMaxGroup];
-    int32_t rb_end[kGemvMaxGroup];
+    const uint8_t* body[NG];  // first block of each packed body
+    const __half* chan_scales[NG];   // per-channel scales (nullptr when grouped)
+    __half* y[NG];            // [M, N_i]
+    int32_t N[NG];
+    int32_t rb_end[NG];
     int32_t n_layers;
     const __half* x;                     // [M, K]
     // Batched form (layers with DIFFERENT inputs in one launch, e.g. the score products of several KV heads): the input
     // of layer i; the plain and grouped forms set every entry to x.  Only the direct form (XDIRECT) reads it per layer.
-    const __half* xl[kGemvMaxGroup];
+    const __half* xl[NG];
     // XSCALE form (the V-cache product of paper Section 3.8): layer i's input is multiplied element-wise by the fp16 vector
     // xscale[i][0 .. K) on its way to the tensor core (x'[m, k] = fp16(x[m, k] * xscale[k])): the per-token scales of a
     // value cache folded into the attention probabilities without a pass of their own.
-    const __half* xscale[kGemvMaxGroup];
+    const __half* xscale[NG];
     int32_t M, K;
     int32_t n_rb;                        // row-blocks holding at least one real row, all layers
     int32_t n_kc;                        // chunks along K
@@ -59,13 +63,14 @@ struct GemvParams {
     int32_t x_bytes;                     // bytes of the x slab (the warp rings follow it)
     int32_t act;                         // gated form only: activation of the gate branch (QL_ACT_*)
 };
+using GemvParams = GemvParamsT<kGemvMaxGroup>;
 
 // GATED: the launch serves exactly two layers of equal shape, gate (0) and up (1), whose row-blocks are dealt out
 // alternately, so that a CTA (which then holds an even number of row-blocks, no cluster) has both branches of
 // every output channel it owns; the epilogue writes y[0] = act(gate) * up (paper Section 3.6: element-wise
 // operators of two branches fused with a fully connected operator).
-template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false>
-__global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams p)
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false, int NG = kGemvMaxGroup>
+__global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT<NG> p)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __half* xs = reinterpret_cast<__half*>(smem_raw);                   // [M][x_stride]
@@ -90,7 +95,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     if (GATED) layer = rb_all & 1;
     else {
 #pragma unroll
-        for (int i = 1; i < kGemvMaxGroup; ++i)
+        for (int i = 1; i < NG; ++i)
             if (i < p.n_layers && rb_all >= p.rb_end[i - 1]) layer = i;
     }
     const int rb = GATED ? rb_all >> 1 : rb_all - (layer ? p.rb_end[layer - 1] : 0);   // row-block inside its layer
@@ -287,7 +292,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParams 
     auto store_out = [&](int rbl, int e, float v) {
         int out_rb = rb_group * rb_per_cta + rbl, ly = 0;
 #pragma unroll
-        for (int i = 1; i < kGemvMaxGroup; ++i)
+        for (int i = 1; i < NG; ++i)
             if (i < p.n_layers && out_rb >= p.rb_end[i - 1]) ly = i;
         out_rb -= ly ? p.rb_end[ly - 1] : 0;
         const int el = e >> 2, i = e & 3;                                // lane that produced it, register index

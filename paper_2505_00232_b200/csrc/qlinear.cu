@@ -224,11 +224,11 @@ cudaError_t ensure_smem_attr(Kern kern, std::atomic<bool>* flags, int device, in
     return e;
 }
 
-template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false>
-cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParams& prm, const GemvPlan& pl, cudaStream_t st)
+template <int BITS, bool GROUPED, bool XDIRECT, bool GATED = false, bool XSCALE = false, int NG = kGemvMaxGroup>
+cudaError_t launch_gemv_x(const qlinear_s* h, const GemvParamsT<NG>& prm, const GemvPlan& pl, cudaStream_t st)
 {
     static std::atomic<bool> attr_set[kMaxDevices];
-    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT, GATED, XSCALE>;
+    auto kern = gemv_kernel<BITS, GROUPED, XDIRECT, GATED, XSCALE, NG>;
     cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, kGemvMaxSmem);
     if (e != cudaSuccess) return e;
     return launch(kern, prm, dim3(pl.grid), dim3(kGemvThreads), pl.smem_bytes, st, pl.cl, h->pdl);
@@ -244,27 +244,20 @@ cudaError_t launch_gemv(const qlinear_s* h, const GemvParams& prm, const GemvPla
     return prm.x_bytes == 0 ? launch_gemv_x<BITS, GROUPED, true>(h, prm, pl, st)
                             : launch_gemv_x<BITS, GROUPED, false>(h, prm, pl, st);
 }
-
-// One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
-// call (integer arithmetic only); nothing is written to a handle.
-// act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
-// xs != nullptr: the batched form, layer i reads xs[i] (x is then ignored); needs the kernel form that reads x straight
-// from global memory.  xscales != nullptr (with xs, int8 layers): layer i's input is multiplied by xscales[i][0 .. K).
-ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1,
-                       const void* const* xs = nullptr, const void* const* xscales = nullptr)
+// The wide form (5 to 8 layers, each with its own input read straight from global memory): int8 layers, the KV heads of
+// an attention layer.
+cudaError_t launch_gemv_wide(const qlinear_s* h, const GemvParamsT<kGemvMaxBatch>& prm, const GemvPlan& pl, cudaStream_t st, bool xscale)
 {
-    const qlinear_s* h = hs[0];
-    const Layout& L = h->L;
-    int n_rb = 0;
-    for (int i = 0; i < n; ++i) n_rb += hs[i]->n_rb;
+    return xscale ? launch_gemv_x<8, false, true, false, true, kGemvMaxBatch>(h, prm, pl, st)
+                  : launch_gemv_x<8, false, true, false, false, kGemvMaxBatch>(h, prm, pl, st);
+}
+
+template <int NG>
+void fill_gemv_params(GemvParamsT<NG>& prm, qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, int n_rb, const GemvPlan& pl,
+                      int act, const void* const* xs, const void* const* xscales)
+{
+    const Layout& L = hs[0]->L;
     const bool gated = act >= 0;
-    if (gated) n_rb = 2 * hs[0]->n_rb;
-    const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
-    if ((gated || xs) && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
-    if (xscales && (!xs || L.bits != 8)) return QL_ERR_UNSUPPORTED;
-    cudaError_t e;
-    if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
-    GemvParams prm{};
     int acc = 0;
     for (int i = 0; i < n; ++i) {
         const Layout& Li = hs[i]->L;
@@ -278,7 +271,7 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     prm.n_layers = n;
     prm.act = gated ? act : 0;
     prm.x = static_cast<const __half*>(xs ? xs[0] : x);
-    for (int i = 0; i < kGemvMaxGroup; ++i) {
+    for (int i = 0; i < NG; ++i) {
         prm.xl[i] = static_cast<const __half*>(xs ? xs[i < n ? i : 0] : x);
         prm.xscale[i] = static_cast<const __half*>(xscales ? xscales[i < n ? i : 0] : nullptr);
     }
@@ -287,6 +280,36 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     prm.n_kc = L.n_kc;
     prm.block_bytes = L.block_bytes;
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
+}
+
+// One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
+// call (integer arithmetic only); nothing is written to a handle.
+// act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
+// xs != nullptr: the batched form, layer i reads xs[i] (x is then ignored); needs the kernel form that reads x straight
+// from global memory; int8 layers may come up to kGemvMaxBatch at a time.  xscales != nullptr (with xs, int8 layers):
+// layer i's input is multiplied by xscales[i][0 .. K).
+ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* ys, int M, cudaStream_t st, int act = -1,
+                       const void* const* xs = nullptr, const void* const* xscales = nullptr)
+{
+    const qlinear_s* h = hs[0];
+    const Layout& L = h->L;
+    int n_rb = 0;
+    for (int i = 0; i < n; ++i) n_rb += hs[i]->n_rb;
+    const bool gated = act >= 0;
+    if (gated) n_rb = 2 * hs[0]->n_rb;
+    const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
+    if ((gated || xs) && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
+    if (xscales && (!xs || L.bits != 8)) return QL_ERR_UNSUPPORTED;
+    if (n > kGemvMaxGroup && (n > kGemvMaxBatch || !xs || L.bits != 8)) return QL_ERR_UNSUPPORTED;
+    cudaError_t e;
+    if (pl.grid <= 0) return QL_ERR_UNSUPPORTED;
+    if (n > kGemvMaxGroup) {
+        GemvParamsT<kGemvMaxBatch> wide{};
+        fill_gemv_params(wide, hs, n, x, ys, M, n_rb, pl, act, xs, xscales);
+        return launch_gemv_wide(h, wide, pl, st, xscales != nullptr) == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+    }
+    GemvParams prm{};
+    fill_gemv_params(prm, hs, n, x, ys, M, n_rb, pl, act, xs, xscales);
     if (L.bits == 8) e = launch_gemv<8, false>(h, prm, pl, st, gated, xscales != nullptr);
     else if (L.grouped) e = launch_gemv<4, true>(h, prm, pl, st, gated);
     else e = launch_gemv<4, false>(h, prm, pl, st, gated);
@@ -546,7 +569,7 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
         if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
         return forward_gemv(const_cast<qlinear_s* const*>(hs), n, x, ys, M, static_cast<cudaStream_t>(stream));
     }
-    if (n > 1 && n <= kGemmMaxGroup && M > hs[0]->gemv_max_m) {          // prefill: one launch of the CTA-pair kernel
+    if (n > 1 && M > hs[0]->gemv_max_m) {                                // prefill: one launch of the CTA-pair kernel
         bool pair_ok = true;
         for (int i = 0; i < n; ++i) pair_ok = pair_ok && (hs[i]->L.n_rsb % 2) == 0 && (gemm_pair_applicable(hs[i]->L, M) || (hs[i]->wmap_ok && gemm_config().ta));
         if (pair_ok) {
@@ -572,7 +595,7 @@ extern "C" ql_status qlinear_forward_group(const qlinear_t* hs, int32_t n, const
 
 extern "C" ql_status qlinear_forward_batch(const qlinear_t* hs, int32_t n, const void* const* xs, void* const* ys, int32_t M, void* stream)
 {
-    if (!hs || !xs || !ys || n < 1 || n > kGemvMaxGroup || M < 1) return QL_ERR_INVALID_ARG;
+    if (!hs || !xs || !ys || n < 1 || n > kGemvMaxBatch || M < 1) return QL_ERR_INVALID_ARG;
     for (int i = 0; i < n; ++i) {
         if (!hs[i] || !xs[i] || !ys[i] || ((reinterpret_cast<uintptr_t>(xs[i]) | reinterpret_cast<uintptr_t>(ys[i])) & 15)) return QL_ERR_INVALID_ARG;
         const Layout &a = hs[0]->L, &b = hs[i]->L;
@@ -764,10 +787,10 @@ extern "C" ql_status qlinear_kv_scores_heads(const qlinear_t* hk, int32_t n_head
         if (!hk[i] || hk[i]->L.bits != 8 || hk[i]->L.N != hk[0]->L.N || hk[i]->L.K != hk[0]->L.K) return QL_ERR_INVALID_ARG;
     const int64_t xs_stride = (int64_t)R * hk[0]->L.K, ys_stride = (int64_t)R * hk[0]->L.N;
     if ((xs_stride | ys_stride) & 7) return QL_ERR_INVALID_ARG;          // every head's rows start on a 16-byte boundary
-    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxGroup) {
-        const int n = std::min(kGemvMaxGroup, n_heads - h0);
-        const void* xs[kGemvMaxGroup];
-        void* ys[kGemvMaxGroup];
+    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxBatch) {
+        const int n = std::min(kGemvMaxBatch, n_heads - h0);
+        const void* xs[kGemvMaxBatch];
+        void* ys[kGemvMaxBatch];
         for (int i = 0; i < n; ++i) {
             xs[i] = static_cast<const __half*>(q_rows) + (h0 + i) * xs_stride;
             ys[i] = static_cast<__half*>(scores) + (h0 + i) * ys_stride;
@@ -794,10 +817,10 @@ extern "C" ql_status qlinear_kv_output_heads(const qlinear_t* hv, int32_t n_head
     if (device_timed_out(hv[0])) return QL_ERR_DEVICE_TIMEOUT;
     DeviceGuard guard(hv[0]->device);
     if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
-    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxGroup) {
-        const int n = std::min(kGemvMaxGroup, n_heads - h0);
-        const void* xs[kGemvMaxGroup];
-        void* ys[kGemvMaxGroup];
+    for (int h0 = 0; h0 < n_heads; h0 += kGemvMaxBatch) {
+        const int n = std::min(kGemvMaxBatch, n_heads - h0);
+        const void* xs[kGemvMaxBatch];
+        void* ys[kGemvMaxBatch];
         for (int i = 0; i < n; ++i) {
             xs[i] = static_cast<const __half*>(prob) + (h0 + i) * xs_stride;
             ys[i] = static_cast<__half*>(out) + (h0 + i) * ys_stride;

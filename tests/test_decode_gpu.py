@@ -227,15 +227,8 @@ def test_forward_group_prefill_and_errors(P, torch):
     other = P.QLinear.from_weights(q8, s8, 8, 0, device="cuda:0")
     with pytest.raises(P.QLinearError):
         P.qlinear_forward_group([lins[0], other], xd)
-    many = (lins * 4)[:8]                                # the most one call takes: prefill size, then one decode launch
-    for lin, y in zip(many, P.qlinear_forward_group(many, xd)):
-        assert torch.equal(y, lin.forward(xd))
-    for i, y in enumerate(P.qlinear_forward_group(many, xd[:4].contiguous())):
-        q, s, _ = cases[i % 2]
-        y64, A, _ = O.linear(x[:4], q, s, 32)
-        assert O.check_against(y.cpu().numpy(), y64, A)[0]
     with pytest.raises(P.QLinearError):
-        P.qlinear_forward_group((lins * 9)[:9], xd)      # more than eight layers
+        P.qlinear_forward_group(lins * 3, xd)            # more than four layers
 
 
 @pytest.mark.parametrize("wi,names,M", [(2, ("q", "k", "v"), 1), (2, ("gate", "up"), 1), (2, ("gate", "up"), 4),
