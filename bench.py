@@ -647,6 +647,7 @@ def main():
                 extra("fused_gating", lambda: gated_record(torch, device, peaks, sidx, ls))
                 extra("residual_rmsnorm", lambda: norm_record(torch, device, peaks, sidx))
                 extra("rope_qkv", lambda: rope_record(torch, device, peaks, sidx))
+                extra("kv_attention", lambda: kv_record(torch, device, peaks, sidx))
                 extra("int8_activations", lambda: a8_record(torch, device, peaks, sidx))
         # ---- CPU oracle beside it (bounded sample)
         if not args.no_cpu_baseline:
@@ -731,6 +732,51 @@ def rope_record(torch, device, peaks, sidx):
         us = ms * 1e3 / (repeats * sets)
         gbs = out["bytes_per_token"] * S / 1e3 / us
         out[stage] = {"S": S, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
+    return out
+
+
+def kv_record(torch, device, peaks, sidx):
+    """The attention products over the KV cache held as weights (paper Section 3.8) for one decode token of a
+    Llama3.1-8B attention layer (8 KV heads of 128, 4 query rows each): append of the token's keys and values, scores
+    and output for all heads, one launch each (the softmax between them is the caller's and not in the region).  At
+    the paper's protocol length (1024 + 256 positions) and at 32768 positions, where the caches of 4 layers (268 MB)
+    are rotated so that they come from HBM."""
+    import paper_2505_00232_b200 as P
+    h_kv, g, d_h = 8, 4, 128
+    rng = np.random.default_rng(5)
+    out = {"h_kv": h_kv, "q_rows_per_head": g, "d_h": d_h, "launches_per_step": 3}
+    for T, layers in ((1280, 4), (32768, 4)):
+        caches = [P.KVHeads(h_kv, T, d_h, device) for _ in range(layers)]
+        kv = torch.from_numpy(rng.standard_normal((h_kv, T, d_h)).astype(np.float16)).to(device)
+        for c in caches:
+            c.append(kv[:, :T - 1].contiguous(), kv[:, :T - 1].contiguous())
+        q = torch.from_numpy(rng.standard_normal((h_kv, g, d_h)).astype(np.float16)).to(device)
+        prob = torch.full((h_kv, g, T), 1.0 / T, dtype=torch.float16, device=device)
+        sc = torch.empty((h_kv, g, T), dtype=torch.float16, device=device)
+        o = torch.empty((h_kv, g, d_h), dtype=torch.float16, device=device)
+        new = kv[:, T - 1:].contiguous()
+
+        def step(i, what=("append", "scores", "output")):
+            c = caches[i % layers]
+            if "append" in what:
+                c.length = T - 1                                          # the same last position every time
+                c.append_raw(new.data_ptr(), new.data_ptr(), d_h, d_h, 1)
+            if "scores" in what:
+                c.scores_raw(q.data_ptr(), sc.data_ptr(), g)
+            if "output" in what:
+                c.output_raw(prob.data_ptr(), o.data_ptr(), g)
+        rec = {"positions": T, "cache_bytes_read": 2 * h_kv * T * d_h}
+        for name, what in (("step", ("append", "scores", "output")), ("append", ("append",)), ("scores", ("scores",)), ("output", ("output",))):
+            graph = capture_graph(torch, lambda i: step(i, what), layers)
+            for _ in range(3):
+                graph.replay()
+            ms, repeats, clocks = timed_region(torch, graph.replay, layers, sidx, 0.2)
+            rec[name + "_us"] = ms * 1e3 / (repeats * layers)
+        rec["gbs"] = rec["cache_bytes_read"] / 1e3 / rec["step_us"]
+        rec["frac_of_measured_peak"] = rec["gbs"] / peaks["hbm_gbs"]
+        out[f"T{T}"] = rec
+        del caches
+        torch.cuda.empty_cache()
     return out
 
 
