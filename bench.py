@@ -637,6 +637,7 @@ def main():
             if not args.no_configs:
                 extra("configs", lambda: decode_configs(torch, device, peaks, sidx, ls, line))
                 extra("decoder_block", lambda: block_record(torch, device, peaks, sidx, ls))
+                extra("launch_floor", lambda: floor_record(torch, sidx, ls))
             # ---- second stage of the hot path on the SAME resident weights (copy 0), measured in the same run
             if not args.no_prefill:
                 extra("prefill", lambda: prefill_sub(torch, device, peaks, args.prefill_steps, sidx, ls.blob0))
@@ -732,6 +733,22 @@ def rope_record(torch, device, peaks, sidx):
         us = ms * 1e3 / (repeats * sets)
         gbs = out["bytes_per_token"] * S / 1e3 / us
         out[stage] = {"S": S, "us": us, "gbs": gbs, "frac_of_measured_peak": gbs / peaks["hbm_gbs"], "sm_mhz": clocks["sm_mhz"]}
+    return out
+
+
+def floor_record(torch, sidx, ls_main):
+    """What a dependent launch costs on this machine: a kernel that does nothing, launched like every kernel of the
+    library, 64 of them chained in a CUDA graph -- one warp, and a grid the size of a decode launch (4 CTAs of 256
+    threads per SM).  The floor under every small layer (config 1 is a single 5.3 MB launch)."""
+    lin = ls_main.lin[0][0]
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    out = {}
+    for name, grid, block in (("one_warp", 1, 32), ("decode_sized_grid", 4 * sms, 256)):
+        graph = capture_graph(torch, lambda i: lin.debug_null_launch(grid, block), 64)
+        for _ in range(3):
+            graph.replay()
+        ms, repeats, clocks = timed_region(torch, graph.replay, 64, sidx, 0.2)
+        out[name + "_us"] = ms * 1e3 / (repeats * 64)
     return out
 
 

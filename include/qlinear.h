@@ -305,6 +305,12 @@ ql_status qlinear_debug_unpack_device(qlinear_t h, int8_t* q_dev_out, void* cuda
  * and the device stays usable.  Asynchronous on `cuda_stream`. */
 ql_status qlinear_debug_expire_wait(qlinear_t h, void* cuda_stream);
 
+/* Measurement aid: launches, the way every kernel of this library is launched (programmatic dependent launch unless
+ * the environment switched it off), a kernel of `grid` blocks of `block` threads that does nothing.  Chained in a
+ * stream or a CUDA graph it gives the cost of a dependent launch on the machine, the floor under every small layer.
+ * Asynchronous on `cuda_stream`. */
+ql_status qlinear_debug_null_launch(qlinear_t h, int32_t grid, int32_t block, void* cuda_stream);
+
 /* Synchronises the handle's device and reports whether any kernel of this library on that device gave up a
  * bounded wait (QL_ERR_DEVICE_TIMEOUT), else QL_OK.  `detail`, if not NULL, receives a code that
  * identifies the wait.  Clears the condition (the flag the forward calls look at, and the arrival counters

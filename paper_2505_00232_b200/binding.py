@@ -23,7 +23,7 @@ ACTIVATIONS = {"identity": QL_ACT_IDENTITY, "silu": QL_ACT_SILU, "gelu_tanh": QL
 
 EXPORTS = (
     "qlinear_packed_size", "qlinear_pack", "qlinear_unpack", "qlinear_create", "qlinear_forward", "qlinear_forward_group", "qlinear_forward_batch", "qlinear_forward_gated", "qlinear_forward_a8", "qlinear_quantize_activations", "qlinear_kv_append", "qlinear_kv_scores", "qlinear_kv_output", "qlinear_kv_append_heads", "qlinear_kv_scores_heads", "qlinear_kv_output_heads", "qlinear_embed", "qlinear_residual_rmsnorm", "qlinear_rope_qkv",
-    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
+    "qlinear_path_for", "qlinear_debug_unpack_device", "qlinear_debug_expire_wait", "qlinear_debug_null_launch", "qlinear_device_status", "qlinear_decode_static", "qlinear_destroy",
     "qlinear_status_string", "qlinear_version", "qlinear_debug_plan", "qlinear_debug_config_reads",
 )
 
@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.qlinear_rope_qkv.restype = ctypes.c_int
     lib.qlinear_debug_expire_wait.argtypes = [vp, vp]
     lib.qlinear_debug_expire_wait.restype = ctypes.c_int
+    lib.qlinear_debug_null_launch.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp]
+    lib.qlinear_debug_null_launch.restype = ctypes.c_int
     pvp = ctypes.POINTER(ctypes.c_void_p)
     lib.qlinear_kv_append_heads.argtypes = [pvp, pvp, ctypes.c_int32, vp, vp, ctypes.c_int64, ctypes.c_int64, pvp, ctypes.c_int32, ctypes.c_int32, vp]
     lib.qlinear_kv_append_heads.restype = ctypes.c_int
@@ -416,6 +418,10 @@ class QLinear:
     def debug_expire_wait(self, stream=None) -> None:
         """Runs the kernels' bounded wait on a barrier nothing completes (about a second); see device_status."""
         _check(lib.qlinear_debug_expire_wait(self._h, _stream_ptr(stream)), "qlinear_debug_expire_wait")
+
+    def debug_null_launch(self, grid: int = 1, block: int = 32, stream=None) -> None:
+        """Launches a kernel that does nothing (what a dependent launch costs on this machine)."""
+        _check(lib.qlinear_debug_null_launch(self._h, grid, block, _stream_ptr(stream)), "qlinear_debug_null_launch")
 
     def device_status(self):
         detail = ctypes.c_uint32(0)

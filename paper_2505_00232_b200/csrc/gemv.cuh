@@ -137,6 +137,32 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
         wsrc += p.block_bytes;
     }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Per-channel scales are weights too: the (at most 4) this thread will apply when it stores outputs are requested
+    // now, so that their latency does not sit at the very end of the kernel.
+    const int t = threadIdx.x;
+    float pre_scale[4] = {1.f, 1.f, 1.f, 1.f};
+    auto out_place = [&](int rbl, int e, int& ly, int& row, int& tok) {  // where element e of the CTA's rbl-th row-block goes
+        int out_rb = rb_group * rb_per_cta + rbl;
+        ly = 0;
+#pragma unroll
+        for (int i = 1; i < NG; ++i)
+            if (i < p.n_layers && out_rb >= p.rb_end[i - 1]) ly = i;
+        out_rb -= ly ? p.rb_end[ly - 1] : 0;
+        const int el = e >> 2, i = e & 3;                                // lane that produced it, register index
+        row = out_rb * kRbRows + (el >> 2) + 8 * (i >> 1);
+        tok = 2 * (el & 3) + (i & 1);
+    };
+    if (!GROUPED && !GATED) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int idx = t + k * kGemvThreads;
+            if (idx < (p.cl > 1 ? 128 : rb_per_cta * 128)) {
+                int ly, row, tok;
+                out_place(idx >> 7, idx & 127, ly, row, tok);
+                if (row < p.N[ly]) pre_scale[k] = __half2float(p.chan_scales[ly][row]);
+            }
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // Stage this CTA's K range of x (zero beyond K) in shared memory -- or, in the direct form, read the
@@ -289,22 +315,15 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
     *reinterpret_cast<float4*>(&red[warp][lane * 4]) = make_float4(total[0], total[1], total[2], total[3]);
     __syncthreads();
 
-    auto store_out = [&](int rbl, int e, float v) {
-        int out_rb = rb_group * rb_per_cta + rbl, ly = 0;
-#pragma unroll
-        for (int i = 1; i < NG; ++i)
-            if (i < p.n_layers && out_rb >= p.rb_end[i - 1]) ly = i;
-        out_rb -= ly ? p.rb_end[ly - 1] : 0;
-        const int el = e >> 2, i = e & 3;                                // lane that produced it, register index
-        const int row = out_rb * kRbRows + (el >> 2) + 8 * (i >> 1);
-        const int tok = 2 * (el & 3) + (i & 1);
+    auto store_out = [&](int rbl, int e, float v, float scale) {
+        int ly, row, tok;
+        out_place(rbl, e, ly, row, tok);
         if (row < p.N[ly] && tok < p.M) {
-            if (!GROUPED) v *= __half2float(p.chan_scales[ly][row]);
+            if (!GROUPED) v *= scale;
             p.y[ly][(int64_t)tok * p.N[ly] + row] = __float2half_rn(v);
         }
     };
 
-    const int t = threadIdx.x;
     if (p.cl > 1) {                                                      // ks_cta == 8: one row-block per CTA
         cg::cluster_group cluster = cg::this_cluster();
         if (t < 128) {
@@ -316,7 +335,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
         if (crank == 0 && t < 128) {
             float v = 0.f;
             for (int r = 0; r < p.cl; ++r) v += *cluster.map_shared_rank(&part[t], r);
-            store_out(0, t, v);
+            store_out(0, t, v, pre_scale[0]);
         }
         cluster.sync();                                                  // peers keep `part` alive until read
     } else if (GATED) {
@@ -333,11 +352,23 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
             }
         }
     } else {
-        for (int idx = t; idx < rb_per_cta * 128; idx += kGemvThreads) {
-            const int rbl = idx >> 7, e = idx & 127;
-            float v = 0.f;
-            for (int s = 0; s < p.ks_cta; ++s) v += red[rbl * p.ks_cta + s][e];
-            store_out(rbl, e, v);
+        if (GROUPED) {
+            for (int idx = t; idx < rb_per_cta * 128; idx += kGemvThreads) {
+                const int rbl = idx >> 7, e = idx & 127;
+                float v = 0.f;
+                for (int s = 0; s < p.ks_cta; ++s) v += red[rbl * p.ks_cta + s][e];
+                store_out(rbl, e, v, 1.f);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {                                // rb_per_cta <= 8: at most 4 elements per thread
+                const int idx = t + k * kGemvThreads;
+                if (idx >= rb_per_cta * 128) break;
+                const int rbl = idx >> 7, e = idx & 127;
+                float v = 0.f;
+                for (int s = 0; s < p.ks_cta; ++s) v += red[rbl * p.ks_cta + s][e];
+                store_out(rbl, e, v, pre_scale[k]);
+            }
         }
     }
 }

@@ -59,8 +59,18 @@ __global__ void __launch_bounds__(kNormThreads) residual_rmsnorm_kernel(const No
     const int n_vec = p.K >> 3;
     constexpr int NV = VPT > 0 ? VPT : 1;
     float keep[NV][8];
-    // programmatic dependent launch: the next kernel may start its own set-up now; x and r may come from the previous one
+    // programmatic dependent launch: the next kernel may start its own set-up now; x and r may come from the previous
+    // one, the weights g do not: they are requested before the wait, so that their latency is not added to the chain
+    // "previous kernel done -> x -> sum -> y" (one token: 2.05 -> 1.6 us)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    uint4 gk[NV];
+    if (VPT > 0) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int v = threadIdx.x + j * kNormThreads;
+            gk[j] = v < n_vec ? *reinterpret_cast<const uint4*>(p.g + 8 * v) : make_uint4(0, 0, 0, 0);
+        }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     auto load_h = [&](int v, float a[8]) {
@@ -103,9 +113,17 @@ __global__ void __launch_bounds__(kNormThreads) residual_rmsnorm_kernel(const No
     __syncthreads();
     const float rstd = rstd_s;
 
-    auto finish = [&](int v, float a[8]) {
+    auto finish = [&](int v, float a[8], const uint4* gv) {
         float g[8];
-        norm_load8(p.g + 8 * v, g);
+        if (gv) {
+            const __half2* h2 = reinterpret_cast<const __half2*>(gv);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h2[i]);
+                g[2 * i] = f.x;
+                g[2 * i + 1] = f.y;
+            }
+        } else norm_load8(p.g + 8 * v, g);
         if (p.h_out) norm_store8(p.h_out + row + 8 * v, a);
 #pragma unroll
         for (int i = 0; i < 8; ++i) a[i] = (a[i] * rstd) * (p.offset + g[i]);
@@ -115,13 +133,13 @@ __global__ void __launch_bounds__(kNormThreads) residual_rmsnorm_kernel(const No
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
             const int v = threadIdx.x + j * kNormThreads;
-            if (v < n_vec) finish(v, keep[j]);
+            if (v < n_vec) finish(v, keep[j], &gk[j]);
         }
     } else {
         for (int v = threadIdx.x; v < n_vec; v += kNormThreads) {
             float a[8];
             load_h(v, a);
-            finish(v, a);
+            finish(v, a, nullptr);
         }
     }
 }

@@ -1068,6 +1068,23 @@ extern "C" ql_status qlinear_decode_static(const qlinear_desc* d, const void* pa
     return QL_OK;
 }
 
+// A kernel that does nothing but take part in programmatic dependent launch: what a launch costs on this machine.
+__global__ void null_kernel(unsigned int* sink)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (sink && threadIdx.x == 0 && blockIdx.x == 0x7fffffff) *sink = 1;   // (never true: keeps the kernel from being empty code)
+}
+
+extern "C" ql_status qlinear_debug_null_launch(qlinear_t h, int32_t grid, int32_t block, void* stream)
+{
+    if (!h || grid < 1 || block < 1 || block > 1024) return QL_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok) { cudaGetLastError(); return QL_ERR_CUDA; }
+    const cudaError_t e = launch(null_kernel, static_cast<unsigned int*>(nullptr), dim3(grid), dim3(block), 0, static_cast<cudaStream_t>(stream), 1, h->pdl);
+    return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+}
+
 extern "C" ql_status qlinear_debug_expire_wait(qlinear_t h, void* stream)
 {
     if (!h) return QL_ERR_INVALID_ARG;
