@@ -26,7 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-Xcompiler", "-fPIC,-O3,-fopenmp", "-shared", "-cudart", "static",
            "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lgomp"]
-    cmd[1:1] = os.environ.get("QL_EXTRA_NVCC_FLAGS", "").split()   # e.g. -DQL_TA_EXPERIMENT for timing experiments
+    cmd[1:1] = os.environ.get("QL_EXTRA_NVCC_FLAGS", "").split()   # extra compiler flags, e.g. -DNAME for an experiment build
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -38,14 +38,6 @@
 #pragma once
 #include "gemm_pair.cuh"
 
-// Build with -DQL_TA_EXPERIMENT to switch parts of the kernel off at run time (timing experiments only: results are
-// then meaningless); without it the switches are compile-time zero.
-#ifdef QL_TA_EXPERIMENT
-#define QL_TA_EXP p.act
-#else
-#define QL_TA_EXP 0
-#endif
-
 namespace ql {
 
 constexpr int kTaFirstDequantWarp = 4;       // warps 4..27: dequantise, six per TMEM lane quarter; 4..19 also run the epilogue
@@ -377,7 +369,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
         if (rank == 0) {
             // f16 x f16 -> f32, both operands K-major (A from tensor memory), M = 256 per pair, N = 256
             // (integer form: u8 weights x s8 activations -> s32)
-            const uint32_t idesc = (I8 ? (2u << 4) | (1u << 10) : (1u << 4)) | ((uint32_t)(((QL_TA_EXP & 256) ? 128 : BN) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+            const uint32_t idesc = (I8 ? (2u << 4) | (1u << 10) : (1u << 4)) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
             const uint32_t b_lo0 = umma_desc_lo(xs_addr(0));
             int s = 0, a = 0;
             uint32_t apar = 0;
@@ -529,7 +521,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                             orow[(cc + 4 * v4 + 2) * 128] = __float2half_rn(f.z * (scale * (float)((int)r[4 * v4 + 2] - OFF * i.z)));
                             orow[(cc + 4 * v4 + 3) * 128] = __float2half_rn(f.w * (scale * (float)((int)r[4 * v4 + 3] - OFF * i.w)));
                         }
-                    } else if (!(QL_TA_EXP & 2)) {
+                    } else {
                         // (the kind of activation is chosen outside the element loop: inside it, the compiler evaluates
                         // every kind and selects)
                         auto store32 = [&](auto f) {
@@ -552,7 +544,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             __syncwarp();
             if (lane == 0) mbar_arrive(grp_bar(wi, 1));
             live = mbar_wait(grp_bar(wi, 1), gpar, abort_flag, 0xC10 + wi) && live;
-            if (live && grp_thread < 64 && m0 + grp_thread < p.M && !(QL_TA_EXP & 2)) {
+            if (live && grp_thread < 64 && m0 + grp_thread < p.M) {
                 const int n0 = rsb * kRsbRows;
                 const uint32_t bytes = (uint32_t)min(kRsbRows, N - n0) * 2;
                 bulk_copy_s2g(p.ly[ly] + (int64_t)(m0 + grp_thread) * N + n0, out_addr + (uint32_t)(64 * wi + grp_thread) * 256, bytes);
@@ -591,11 +583,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             // producer issues the load of step g only after step g - NW's warps have released the stage: wait for that first.
             if (NW % 3 != 0 && !mbar_wait(wempty_bar(s), wpar ^ 1, abort_flag, 0x480 + s)) { ok = false; break; }
             if (!mbar_wait(wfull_bar(s), wpar, abort_flag, 0x400 + s)) { ok = false; break; }
-            if (!(QL_TA_EXP & 4)) dq.template convert<BITS, GROUPED, I8>(wpk_addr(s), half, r);
-            else {
-#pragma unroll
-                for (int i = 0; i < 16; ++i) r[i] = 0;
-            }
+            dq.template convert<BITS, GROUPED, I8>(wpk_addr(s), half, r);
             // the MMAs that read slot a (step g - NA) have retired
             if (!mbar_wait(aempty_bar(a), apar, abort_flag, 0xB00 + a)) { ok = false; break; }
             tc_fence_after();
@@ -669,9 +657,6 @@ ql_status gemm_pair_ta_launch(const GemmPairLayers& set, const void* x, int M, c
     }
     prm.n_layers = set.n;
     prm.act = act;
-#ifdef QL_TA_EXPERIMENT
-    if (!GATED) prm.act = getenv("QLINEAR_EXP") ? atoi(getenv("QLINEAR_EXP")) : 0;
-#endif
     if (GATED) n_rsb = L.n_rsb;                                          // work units count positions of one layer
     prm.M = M; prm.N = L.N; prm.K = L.K;
     prm.n_kc = L.n_kc; prm.block_bytes = L.block_bytes;
