@@ -238,7 +238,9 @@ ql_status qlinear_kv_output(qlinear_t h_v, const void* prob_dev, const void* v_s
  *                            there is no scratch buffer and no pass of its own.  Other shapes: QL_ERR_UNSUPPORTED
  *                            (use qlinear_kv_output per head).
  * All device pointers 16-byte aligned, R * d_h and R * cache positions multiples of 8.  Results are bit-identical to
- * the per-head calls.  Asynchronous, allocate nothing.  Errors as above. */
+ * the per-head calls wherever those take K undivided (d_h <= 128) and meet the same tolerance everywhere.  Score
+ * products of more than four row super-blocks per SM (long caches; R <= 8, d_h = 64, 128 or 256) run on a persistent
+ * kernel of their own (csrc/gemv_rows.cuh).  Asynchronous, allocate nothing.  Errors as above. */
 ql_status qlinear_kv_append_heads(const qlinear_t* h_k, const qlinear_t* h_v, int32_t n_heads, const void* k_new_dev,
                                   const void* v_new_dev, int64_t head_stride, int64_t token_stride, void* const* v_scale_dev,
                                   int32_t pos, int32_t n_new, void* cuda_stream);

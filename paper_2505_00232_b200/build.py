@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libqlinear.so")
 SOURCES = ["qlinear.cu", "pack.cpp"]
-DEPS = SOURCES + ["layout.h", "dequant.cuh", "sm100_ptx.cuh", "embed.cuh", "gemv.cuh", "gemv_a8.cuh", "kv.cuh", "gemv_stream.cuh", "gemm.cuh", "gemm_pair.cuh", "gemm_pair_ta.cuh", "norm.cuh", "rope.cuh", os.path.join("..", "..", "include", "qlinear.h")]
+DEPS = SOURCES + ["layout.h", "dequant.cuh", "sm100_ptx.cuh", "embed.cuh", "gemv.cuh", "gemv_rows.cuh", "gemv_a8.cuh", "kv.cuh", "gemv_stream.cuh", "gemm.cuh", "gemm_pair.cuh", "gemm_pair_ta.cuh", "norm.cuh", "rope.cuh", os.path.join("..", "..", "include", "qlinear.h")]
 
 
 def _stale() -> bool:

@@ -25,6 +25,7 @@ __device__ unsigned int* g_status_host;
 #include "dequant.cuh"
 #include "embed.cuh"
 #include "gemv.cuh"
+#include "gemv_rows.cuh"
 #include "gemv_stream.cuh"
 #include "gemv_a8.cuh"
 #include "kv.cuh"
@@ -282,6 +283,19 @@ void fill_gemv_params(GemvParamsT<NG>& prm, qlinear_s* const* hs, int n, const v
     prm.ks_cta = pl.ks_cta; prm.ks_cta_log2 = pl.ks_cta == 8 ? 3 : pl.ks_cta == 4 ? 2 : pl.ks_cta == 2 ? 1 : 0; prm.cl = pl.cl; prm.cps = pl.cps; prm.x_stride = pl.x_stride; prm.x_bytes = pl.x_bytes;
 }
 
+// The persistent form for int8 layers with many rows and a short K (gemv_rows.cuh): every layer with its own input.
+template <int NKC>
+cudaError_t launch_gemv_rows(const qlinear_s* h, const GemvRowsParams& prm, cudaStream_t st)
+{
+    static std::atomic<bool> attr_set[kMaxDevices];
+    auto kern = gemv_rows_kernel<NKC>;
+    const int smem = kGemvWarps * 2 * NKC * 512;
+    cudaError_t e = ensure_smem_attr(kern, attr_set, h->device, smem);
+    if (e != cudaSuccess) return e;
+    const int grid = std::min(prm.n_rsb, h->num_sms * (NKC <= 4 ? 4 : 3));
+    return launch(kern, prm, dim3(grid), dim3(kGemvThreads), smem, st, 1, h->pdl);
+}
+
 // One launch for n layers that read the same x (n == 1: the plain forward).  The plan of a group is made per
 // call (integer arithmetic only); nothing is written to a handle.
 // act >= 0: the gated form (n == 2: gate, up; ys[0] the output; the row-blocks of the two layers alternate).
@@ -297,6 +311,26 @@ ql_status forward_gemv(qlinear_s* const* hs, int n, const void* x, void* const* 
     for (int i = 0; i < n; ++i) n_rb += hs[i]->n_rb;
     const bool gated = act >= 0;
     if (gated) n_rb = 2 * hs[0]->n_rb;
+    // many rows, short K (the score product over a long KV cache): more than one wave of row super-blocks
+    if (xs && !xscales && !gated && n <= kGemvMaxBatch && L.bits == 8 && (L.K % 32) == 0 && (L.n_kc == 2 || L.n_kc == 4 || L.n_kc == 8)) {
+        GemvRowsParams rp{};
+        int n_rsb = 0;
+        for (int i = 0; i < n; ++i) {
+            const Layout& Li = hs[i]->L;
+            rp.body[i] = hs[i]->blob + Li.body_offset;
+            rp.chan_scales[i] = reinterpret_cast<const __half*>(hs[i]->blob + Li.chan_scale_offset);
+            rp.y[i] = static_cast<__half*>(ys[i]);
+            rp.xl[i] = static_cast<const __half*>(xs[i]);
+            rp.N[i] = Li.N;
+            n_rsb += Li.n_rsb;
+            rp.rsb_end[i] = n_rsb;
+        }
+        if (n_rsb > 4 * h->num_sms) {
+            rp.n_layers = n; rp.M = M; rp.K = L.K; rp.n_rsb = n_rsb; rp.block_bytes = L.block_bytes;
+            const cudaError_t e = L.n_kc == 2 ? launch_gemv_rows<2>(h, rp, st) : L.n_kc == 4 ? launch_gemv_rows<4>(h, rp, st) : launch_gemv_rows<8>(h, rp, st);
+            return e == cudaSuccess ? QL_OK : QL_ERR_CUDA;
+        }
+    }
     const GemvPlan pl = gated ? plan_gemv(L, n_rb, M, h->num_sms, true) : n == 1 ? h->gemv[M] : plan_gemv(L, n_rb, M, h->num_sms);
     if ((gated || xs) && (pl.grid <= 0 || pl.x_bytes != 0)) return QL_ERR_UNSUPPORTED;
     if (xscales && (!xs || L.bits != 8)) return QL_ERR_UNSUPPORTED;

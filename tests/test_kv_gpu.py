@@ -139,3 +139,29 @@ def test_heads_argument_errors(P, torch):
         heads.output(big)                               # 9 query rows: not a decode-sized product
     with pytest.raises(P.QLinearError):
         heads.append(torch.zeros((3, 1, 64), dtype=torch.float16, device="cuda"), torch.zeros((3, 1, 64), dtype=torch.float16, device="cuda"))
+
+
+@pytest.mark.parametrize("d_h,cache,n_heads,R", [(128, 10240, 8, 4), (64, 20000 // 32 * 32, 8, 1), (256, 9632, 8, 8), (128, 25632, 3, 5)],
+                         ids=["dh128", "dh64-one-row", "dh256-eight-rows", "three-heads-ragged"])
+def test_scores_over_a_long_cache_match_the_per_head_calls(P, torch, d_h, cache, n_heads, R):
+    """More than one wave of row super-blocks: the score product of all heads runs on the persistent short-K kernel
+    (a CTA walks over super-blocks, the next one's bytes in flight).  Same bits as the per-head calls of the ordinary
+    decode kernel; cache lengths that are not a multiple of 128; positions beyond the filled part score 0."""
+    T = cache - 777
+    rng = np.random.default_rng(d_h + cache)
+    k = (rng.standard_normal((n_heads, T, d_h)) * rng.uniform(0.2, 3.0, size=(n_heads, T, 1))).astype(np.float16)
+    q = rng.standard_normal((n_heads, R, d_h)).astype(np.float16)
+    kd, qd = torch.from_numpy(k).cuda(), torch.from_numpy(q).cuda()
+    heads = P.KVHeads(n_heads, cache, d_h)
+    heads.append(kd, kd)
+    sc = heads.scores(qd)
+    torch.cuda.synchronize()
+    assert heads.heads[0].k.device_status() == (0, 0)
+    assert (sc[:, :, T:] == 0).all()
+    for h in range(n_heads):
+        if d_h <= 128:                                  # (at d_h = 256 the per-head call splits K: another order of sums)
+            assert torch.equal(sc[h], heads.heads[h].scores(qd[h]))
+        k_q, k_s = O.kv_quantize_rows(k[h])
+        y64, A, _ = O.linear(q[h], k_q, k_s.reshape(-1, 1), 0)
+        ok, rel, worst = O.check_against(sc[h, :, :T].cpu().numpy(), y64, A)
+        assert ok, (h, rel, worst)
