@@ -173,6 +173,9 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = f
             // slices on half as many warps)
             double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 4 ? 1.25 : 0.0) - (cps < 2 ? 1.0 : 0.0);
             if (warps > target) score -= 2.0;                               // more CTAs than fit at once: a second wave
+            // a cluster launch and its two cluster-wide barriers cost about a microsecond: more than a launch of a few MB
+            // gains from the extra warps (V-cache product of 8 heads at 1280 positions: 4.2 us with clusters of 5, 3.1 us without)
+            if (cl > 1 && (double)n_rb * L.n_kc * 512.0 < 4.0e6) score -= 0.75;
             if (cfg.force_ks && !gated) score = (ks == cfg.force_ks) ? 0.0 : -1e29;
             if (score > best_score) {
                 best_score = score;
