@@ -510,6 +510,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-workload record (configs 1-5, LM head, q8, 8/4/4)")
     ap.add_argument("--prefill-steps", type=int, default=20)
+    ap.add_argument("--records", default="", help="comma-separated names of the auxiliary records to run (default: all), e.g. kv_attention")
     ap.add_argument("--quick", action="store_true",
                     help="main timed region only (no e2e, per-kernel, prefill or CPU legs): the command to profile")
     args = ap.parse_args()
@@ -621,8 +622,12 @@ def main():
     }
 
     if rank == 0 and world == 1:
+        wanted = {r for r in args.records.split(",") if r}
+
         def extra(name, fn, append=False):
             """An auxiliary record must not cost the line: on failure its place holds the error."""
+            if wanted and name not in wanted:
+                return
             try:
                 rec = fn()
                 line[name] = line[name] + rec if append else rec
@@ -643,7 +648,7 @@ def main():
                 extra("prefill", lambda: prefill_sub(torch, device, peaks, args.prefill_steps, sidx, ls.blob0))
             if not args.no_configs:
                 if not isinstance(line.get("configs"), list):
-                    line["configs"] = [line["configs"]]
+                    line["configs"] = [line["configs"]] if "configs" in line else []
                 extra("configs", lambda: prefill_configs(torch, device, peaks, sidx, line), append=True)
                 extra("fused_gating", lambda: gated_record(torch, device, peaks, sidx, ls))
                 extra("residual_rmsnorm", lambda: norm_record(torch, device, peaks, sidx))
