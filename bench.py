@@ -462,7 +462,11 @@ def prefill_roofline(torch, ls, workload, M, peaks, sampler_index, kernel_name="
     return {"bound": "tensor", "kernel": kernel_name + ": the int4 layers as single launches, average", "achieved": ach,
             "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
             "traffic": NCU_TRAFFIC_BYTES.get((workload.name, M)), "peak_source": peaks["source"],
-            "flops_per_launch": flops, "us_per_launch": ms * 1e3, "frac_of_nominal_2250": ach / 2250.0}
+            "flops_per_launch": flops, "us_per_launch": ms * 1e3, "frac_of_nominal_2250": ach / 2250.0,
+            # the launches are timed back to back for at least a quarter of a second, i.e. under the power limit: next to
+            # the burst peak (the denominator of `frac`) the peak of a seconds-long cuBLAS loop on the same part
+            "peak_sustained": peaks.get("bf16_tflops_sustained"),
+            "frac_of_sustained_peak": ach / peaks["bf16_tflops_sustained"] if peaks.get("bf16_tflops_sustained") else None}
 
 
 def config_entry(torch, device, peaks, sampler_index, name, M, copies=0, blobs=None, ls=None, steps=0):
