@@ -216,7 +216,7 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Pa
     float ftotal[4] = {0.f, 0.f, 0.f, 0.f};                              // GROUPED: sum_g s * acc, fp32
     int itotal[4] = {0, 0, 0, 0};                                        // per channel: the integer sum (offset term added below)
     const signed char* xrow = xq + min(g, p.M - 1) * p.xq_stride + 8 * c;   // columns g >= M copy the last token, never stored
-    const uint32_t sc_u32 = sbuf_u32 - lane * 16 + g * 8;
+    [[maybe_unused]] const uint32_t sc_u32 = sbuf_u32 - lane * 16 + g * 8;   // (read by the grouped form only)
     int sflip = 0;
     for (int kc = kc0; kc < kc1; kc += kGemvRing) {
 #pragma unroll
