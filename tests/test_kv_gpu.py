@@ -165,3 +165,18 @@ def test_scores_over_a_long_cache_match_the_per_head_calls(P, torch, d_h, cache,
         y64, A, _ = O.linear(q[h], k_q, k_s.reshape(-1, 1), 0)
         ok, rel, worst = O.check_against(sc[h, :, :T].cpu().numpy(), y64, A)
         assert ok, (h, rel, worst)
+
+
+def test_small_launches_are_planned_without_clusters(P, torch):
+    """A cluster launch with its cluster-wide barriers costs about a microsecond: launches of a few MB (the V-cache
+    product at the protocol length) are planned without one, large layers with a long K still take clusters."""
+    import ctypes
+
+    def plan(lin, M):
+        out = (ctypes.c_int32 * 8)()
+        assert P.lib.qlinear_debug_plan(lin._h, M, out, 8) == 8
+        return {"grid": out[1], "cl": out[2], "ks_cta": out[3], "cps": out[4]}
+    v = P.KVCache(CACHE, DH).v                           # N = 128, K = 1280: 164 KB
+    assert plan(v, 4)["cl"] == 1
+    big = P.QLinear(P.Desc(4096, 14336, 8, 0), torch.zeros(P.qlinear_packed_size(P.Desc(4096, 14336, 8, 0)), dtype=torch.uint8, device="cuda"))
+    assert plan(big, 1)["cl"] > 1
