@@ -50,6 +50,7 @@ struct Config {
     int gemv_max_m;          // QLINEAR_GEMV_MAX_M: largest M served by the decode kernels (1..8)
     bool pdl;                // QLINEAR_PDL: programmatic dependent launch attribute on every kernel
     int warps_per_sm;        // QLINEAR_GEMV_WARPS_PER_SM: residency target of the cluster decode kernel
+    bool oversubscribe;      // QLINEAR_GEMV_OVERSUBSCRIBE=0: the group-scaled int4 decode kernel never takes more CTAs than fit at once
     int force_ks;            // QLINEAR_GEMV_KS: forced K split of the cluster decode kernel (0 = planned)
     bool xdirect;            // QLINEAR_GEMV_XDIRECT: x fragments straight from global memory
     int kernel;              // QLINEAR_GEMV_KERNEL: 0 / 1 cluster kernel (default), 2 streaming kernel
@@ -67,6 +68,7 @@ void load_config()
     c.gemv_max_m = std::max(1, std::min(8, env_int("QLINEAR_GEMV_MAX_M", 8)));
     c.pdl = env_int("QLINEAR_PDL", 1) != 0;
     c.warps_per_sm = env_int("QLINEAR_GEMV_WARPS_PER_SM", 32);
+    c.oversubscribe = env_int("QLINEAR_GEMV_OVERSUBSCRIBE", 1) != 0;
     c.force_ks = env_int("QLINEAR_GEMV_KS", 0);
     c.xdirect = env_int("QLINEAR_GEMV_XDIRECT", 1) != 0;
     const char* kc = std::getenv("QLINEAR_GEMV_KERNEL");
@@ -172,7 +174,13 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = f
             // slices of fewer than 4 chunks never reach a steady state (measured: 2-chunk slices lose to 4-chunk
             // slices on half as many warps)
             double score = -std::fabs(std::log2(warps / target)) + 2.0 * std::log2(eff) - (cps < 4 ? 1.25 : 0.0) - (cps < 2 ? 1.0 : 0.0);
-            if (warps > target) score -= 2.0;                               // more CTAs than fit at once: a second wave
+            // More CTAs than fit at once mean a second wave -- except, for the group-scaled int4 kernel (bound by its
+            // instruction stream, not by the memory system) at one token, up to about one and a half waves of CTAs without
+            // clusters whose slices stay long: the partial second wave fills in as the first one drains, and the finer
+            // units even out the end (Llama gate + up: 17.8 us with 0.76 of a wave, 17.2 us with 1.5 waves).  Measured limits
+            // of the rule: the int8 and per-channel forms of the same launch lose 2 to 7 % that way, and with 2 to 8 tokens
+            // the launch itself still gains but the step that contains it loses 1 to 3 % (the next launch gets its SMs later).
+            if (warps > target) score += (cfg.oversubscribe && M == 1 && L.grouped && cl == 1 && warps <= 1.55 * target && cps >= 16) ? 0.25 : -2.0;
             // a cluster launch and its two cluster-wide barriers cost about a microsecond: more than a launch of a few MB
             // gains from the extra warps (V-cache product of 8 heads at 1280 positions: 4.2 us with clusters of 5, 3.1 us without)
             if (cl > 1 && (double)n_rb * L.n_kc * 512.0 < 4.0e6) score -= 0.75;
