@@ -181,9 +181,12 @@ GemvPlan plan_gemv(const Layout& L, int n_rb, int M, int num_sms, bool gated = f
             // of the rule: the int8 and per-channel forms of the same launch lose 2 to 7 % that way, and with 2 to 8 tokens
             // the launch itself still gains but the step that contains it loses 1 to 3 % (the next launch gets its SMs later).
             if (warps > target) score += (cfg.oversubscribe && M == 1 && L.grouped && cl == 1 && warps <= 1.55 * target && cps >= 16) ? 0.25 : -2.0;
-            // a cluster launch and its two cluster-wide barriers cost about a microsecond: more than a launch of a few MB
-            // gains from the extra warps (V-cache product of 8 heads at 1280 positions: 4.2 us with clusters of 5, 3.1 us without)
-            if (cl > 1 && (double)n_rb * L.n_kc * 512.0 < 4.0e6) score -= 0.75;
+            // a cluster launch and its two cluster-wide barriers cost a microsecond or two (the CTAs of a cluster start
+            // together and leave together): more than a launch of a few MB gains from the extra warps (V-cache product of 8
+            // heads at 1280 positions: 4.2 us with clusters of 5, 3.1 us without; one 2304 x 2304 int8 layer: 4.0 / 3.7 us).
+            // Larger launches keep their clusters: timed alone they look better without (Llama o, 16.8 MB: 5.9 / 4.6 us),
+            // but inside the step the under-filled grid costs the launches around it more than it saves.
+            if (cl > 1 && (double)n_rb * L.n_kc * 512.0 < 6.0e6) score -= 0.75;
             if (cfg.force_ks && !gated) score = (ks == cfg.force_ks) ? 0.0 : -1e29;
             if (score > best_score) {
                 best_score = score;
