@@ -445,7 +445,7 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
             __threadfence();
             __syncwarp();
             unsigned int old = 0;
-            if (lane == 0) { mbar_arrive_remote(tempty_bar, 0); old = atomicAdd(cnt, 1u); }
+            if (lane == 0) { mbar_arrive_remote_relaxed(tempty_bar, 0); old = atomicAdd(cnt, 1u); }
             old = __shfl_sync(0xffffffffu, old, 0);
             if ((int)old != P - 1) return;
             __threadfence();
@@ -504,9 +504,13 @@ gemm_pair_ta_kernel(const __grid_constant__ TaMaps maps, const GemmParams p)
                     uint32_t r[32];
                     tmem_ld32(taddr + (uint32_t)cc, r);
                     if (cc == 32) {                                      // accumulator read: the next tile's MMAs may start
+                        // RELAXED arrive, like the relay's: what must precede the leader's next MMA is the completion of
+                        // this warp's tensor-memory loads, which tcgen05.wait::ld (inside tmem_ld32) has already waited
+                        // for; nothing in shared or global memory is handed over.  With release semantics at cluster
+                        // scope the arrive sat on the critical path of every tile boundary (Llama gate: 179 -> 176 us).
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive_remote(tempty_bar, 0);
+                        if (lane == 0) mbar_arrive_remote_relaxed(tempty_bar, 0);
                     }
                     if (I8) {
                         // acc = sum (q + off) * xq: remove off * (sum of the token's quantised row), then both scales; the 32
