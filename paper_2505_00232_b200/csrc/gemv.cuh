@@ -337,7 +337,9 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
             for (int r = 0; r < p.cl; ++r) v += *cluster.map_shared_rank(&part[t], r);
             store_out(0, t, v, pre_scale[0]);
         }
-        cluster.sync();                                                  // peers keep `part` alive until read
+        // peers keep `part` alive until it has been read: a rendezvous only, nothing is handed over, so the arrive
+        // needs no release and the wait no acquire
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
     } else if (GATED) {
         for (int idx = t; idx < (rb_per_cta >> 1) * 128; idx += kGemvThreads) {
             const int pr = idx >> 7, e = idx & 127;                      // pair of row-blocks (gate, up), element
