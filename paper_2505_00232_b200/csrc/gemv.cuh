@@ -331,7 +331,10 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_kernel(const GemvParamsT
             for (int s = 0; s < kGemvWarps; ++s) v += red[s][t];
             part[t] = v;
         }
-        cluster.sync();
+        // partial sums published to the cluster: every CTA releases, only the reading CTA has to acquire
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        if (crank == 0) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        else asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
         if (crank == 0 && t < 128) {
             float v = 0.f;
             for (int r = 0; r < p.cl; ++r) v += *cluster.map_shared_rank(&part[t], r);

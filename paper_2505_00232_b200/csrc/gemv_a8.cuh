@@ -318,7 +318,8 @@ __global__ void __launch_bounds__(kGemvThreads, 4) gemv_a8_kernel(const GemvA8Pa
             for (int r = 0; r < p.cl; ++r) add(f, i, *cluster.map_shared_rank(&part[t], r));
             store_out(0, t, f, i);
         }
-        cluster.sync();                                                  // peers keep `part` alive until read
+        // peers keep `part` alive until it has been read: a rendezvous only (relaxed arrive, plain wait)
+        asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
     } else {
         for (int idx = t; idx < rb_per_cta * 128; idx += kGemvThreads) {
             const int rbl = idx >> 7, e = idx & 127;
