@@ -27,7 +27,10 @@
 // What bounded it (measured): not the tensor pipe (halving the MMA width changed nothing) but the instruction stream
 // of the dequantise warps and of the polling threads around them, which is why every warp loops over its own steps
 // only and no thread polls in the main loop.  As it stands the tensor pipe is active 86-91 % of the cycles in which an
-// SM has work, at the clock the power limit leaves.
+// SM has work (tiles of 64 k-steps; 71 % with 36), at the clock the power limit leaves: what is missing is a constant
+// 3-4 us per tile boundary -- last MMAs retire, epilogue warps finish their step, meet, take the accumulator out, tell
+// the leader across the SM pair -- which is why both cross-SM signals on that path (the relay's and the epilogue's)
+// are relaxed arrives.
 //
 // Forms of the kernel (template flags): the plain product, whole tiles dealt out round-robin or, for launches with
 // few tiles, 2 or 4 K parts per tile that meet in the device scratch; GATED (y = act(gate) * up, Section 3.6); I8
